@@ -1,0 +1,91 @@
+"""Eq. 2 and Eq. 4 of the paper in exact rational arithmetic.  TEST INFRASTRUCTURE ONLY.
+
+Pure Python ``fractions.Fraction``: slow, for small cases.  It is written from the
+formulas as printed (e, m, R_OF, R_UF, the three cases), not from the C++ oracle, and the
+two are compared in the tests.  A format is ``(M, E, b, rounding, flags)``.
+"""
+from fractions import Fraction
+import math
+
+
+def decode_e4m3(code: int) -> Fraction:
+    """Value of an OCP E4M3 byte: sign, 4 exponent bits (bias 7), 3 mantissa bits."""
+    s, e, f = code >> 7, (code >> 3) & 15, code & 7
+    if e == 15 and f == 7:
+        raise ValueError("E4M3 NaN code")
+    if e == 0:
+        v = Fraction(f, 8) * Fraction(1, 2 ** 6)
+    else:
+        v = (1 + Fraction(f, 8)) * Fraction(2) ** (e - 7)
+    return -v if s else v
+
+
+def r_of(M, E, b) -> Fraction:
+    return Fraction(2) ** (2 ** E - b - 1) * (2 - Fraction(1, 2 ** M))
+
+
+def r_uf(b) -> Fraction:
+    return Fraction(2) ** (-b)
+
+
+def _floor_log2(a: Fraction) -> int:
+    # a > 0 ; exact: compare integers, never floats
+    e = a.numerator.bit_length() - a.denominator.bit_length()
+    if Fraction(2) ** e > a:
+        e -= 1
+    elif Fraction(2) ** (e + 1) <= a:
+        e += 1
+    assert Fraction(2) ** e <= a < Fraction(2) ** (e + 1)
+    return e
+
+
+def _round(v: Fraction, nearest: bool) -> int:
+    fl = math.floor(v)
+    if not nearest:
+        return fl
+    rem = v - fl
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2 == 1):
+        return fl + 1
+    return fl
+
+
+def quantise(fmt, x) -> Fraction:
+    """Q^FLOAT_{M,E,b}(x), Eq. 2, cases in the printed order; zero is +0."""
+    M, E, b, rounding, flags = fmt
+    x = Fraction(x)
+    if x == 0:
+        return Fraction(0)
+    sign = -1 if x < 0 else 1
+    a = abs(x)
+    top = r_of(M, E, b)
+    if a >= top:
+        return sign * top
+    if (flags & 1) and a < r_uf(b):
+        return Fraction(0)
+    e = _floor_log2(a)
+    m = Fraction(_round(Fraction(2) ** M * (a / Fraction(2) ** e - 1), rounding == 1), 2 ** M)
+    y = Fraction(2) ** e * (m + 1)
+    return sign * min(y, top)
+
+
+def fmaq(prod_fmt, acc_fmt, x: Fraction, w: Fraction, s: Fraction) -> Fraction:
+    """Eq. 4."""
+    return quantise(acc_fmt, quantise(prod_fmt, x * w) + s)
+
+
+def dot(prod_fmt, acc_fmt, order, chunk, xcodes, wcodes) -> Fraction:
+    """Eq. 8-9 (order 0) or two-hierarchy chunked accumulation (order 1) over byte codes."""
+    xs = [decode_e4m3(int(c)) for c in xcodes]
+    ws = [decode_e4m3(int(c)) for c in wcodes]
+    if order == 0:
+        s = Fraction(0)
+        for x, w in zip(xs, ws):
+            s = fmaq(prod_fmt, acc_fmt, x, w, s)
+        return s
+    total = Fraction(0)
+    for j in range(0, len(xs), chunk):
+        c = Fraction(0)
+        for x, w in zip(xs[j:j + chunk], ws[j:j + chunk]):
+            c = fmaq(prod_fmt, acc_fmt, x, w, c)
+        total = quantise(acc_fmt, c + total)
+    return total

@@ -1,0 +1,54 @@
+"""Format descriptors for Q_prod and Q_acc (Eq. 2 of the paper) and the bias rules used by the harness."""
+from dataclasses import dataclass
+
+ROUND_FLOOR = 0          # floor on the magnitude: the paper's choice (Sec. 3)
+ROUND_NEAREST_EVEN = 1   # a parameter of the benchmark's format sweep, not the paper's choice
+FLAG_UNDERFLOW = 1       # bit0 of flags: the |x| < R_UF -> 0 branch of Eq. 2 is active
+
+ORDER_SEQUENTIAL = 0     # Eq. 8-9
+ORDER_CHUNKED = 1        # two hierarchies, Sec. 3 / App. D
+PAPER_CHUNK = 16         # "constant chunk size of 16" (Sec. 3)
+
+
+@dataclass(frozen=True)
+class LbaFormat:
+    """Q^FLOAT_{M,E,b}: M mantissa bits, E exponent bits, exponent bias b, rounding, flags."""
+    man_bits: int
+    exp_bits: int
+    bias: int
+    rounding: int = ROUND_FLOOR
+    flags: int = FLAG_UNDERFLOW
+
+    def as_tuple(self):
+        return (self.man_bits, self.exp_bits, self.bias, self.rounding, self.flags)
+
+    @property
+    def r_uf(self) -> float:
+        return 2.0 ** (-self.bias)
+
+    @property
+    def r_of(self) -> float:
+        return 2.0 ** (2 ** self.exp_bits - self.bias - 1) * (2.0 - 2.0 ** (-self.man_bits))
+
+
+def code_domain_formats(man_bits: int = 7, exp_bits: int = 4, rounding: int = ROUND_FLOOR,
+                        flags: int = FLAG_UNDERFLOW, chunk: int = PAPER_CHUNK):
+    """(prod_fmt, acc_fmt) for FMAq on raw E4M3 code values.
+
+    b_prod is the largest integer bias for which the largest code product, 448^2, stays
+    below R_OF (the paper's flex-bias rule of Sec. 3.1 applied to products): 2^E - 18.
+    b_acc = b_prod - log2(chunk)/2 (Sec. 3, the chunk-size rule; 2 for chunk 16).
+    """
+    b_prod = 2 ** exp_bits - 18
+    half_log = 0
+    c = chunk
+    while c >= 4:
+        half_log += 1
+        c //= 4
+    prod = LbaFormat(man_bits, exp_bits, b_prod, rounding, flags)
+    acc = LbaFormat(man_bits, exp_bits, b_prod - half_log, rounding, flags)
+    return prod, acc
+
+
+M7E4_PAPER = (LbaFormat(7, 4, 12), LbaFormat(7, 4, 10))   # real-domain biases of the ResNet runs (Sec. 3.1)
+WIDE = LbaFormat(23, 8, 127)                               # binary32-like: nothing in Eq. 2 is reachable

@@ -1,0 +1,196 @@
+"""Pins for the oracle's FMAq chain (Eq. 4, Eq. 8-9, chunked accumulation).  CPU only."""
+import ctypes
+import os
+import subprocess
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import lba_oracle as orc
+from oracle import lba_exact as ex
+from paper_2401_14110_b200 import synth
+
+SEQ, CHK = orc.SEQUENTIAL, orc.CHUNKED
+WIDE_NEAREST = (23, 8, 127, 1, 1)
+WIDE_FLOOR = (23, 8, 127, 0, 1)
+FINITE = np.array([c for c in range(256) if (c & 0x7F) != 0x7F], dtype=np.uint8)
+
+
+def _decode_f32(codes):
+    return synth.e4m3_decode(torch.from_numpy(np.ascontiguousarray(codes))).numpy()
+
+
+def test_decode_matches_pytorch_float8_cast():
+    vals = _decode_f32(FINITE)
+    for c, v in zip(FINITE, vals):
+        assert orc.decode_e4m3(int(c)) == float(v)
+        assert ex.decode_e4m3(int(c)) == Fraction(float(v))
+    assert orc.decode_e4m3(0x7E) == 448.0 and orc.decode_e4m3(0x01) == 2.0 ** -9
+    for nan_code in (0x7F, 0xFF):
+        with pytest.raises(orc.OracleError):
+            orc.decode_e4m3(nan_code)
+
+
+def test_hand_worked_chains(golden_dir):
+    n = 0
+    with open(os.path.join(golden_dir, "fmaq_chains.txt")) as fh:
+        for line in fh:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            name, rnd, order, chunk, K, xb, wb, want, *sums = line.split()
+            rnd, order, chunk, K = int(rnd), int(order), int(chunk), int(K)
+            prod, acc = (7, 4, 12, rnd, 1), (7, 4, 10, rnd, 1)
+            x = np.full(K, int(xb, 16), np.uint8)
+            w = np.full(K, int(wb, 16), np.uint8)
+            y, tr = orc.dot(prod, acc, order, chunk, x, w, trace=True)
+            assert y == float(want), name
+            if sums:
+                assert list(tr) == [float(v) for v in sums], name
+            assert ex.dot(prod, acc, order, chunk, x, w) == Fraction(float(want)), name
+            n += 1
+    assert n == 6
+
+
+@pytest.fixture(scope="module")
+def fp32_chain(tmp_path_factory):
+    src = os.path.join(os.path.dirname(__file__), "helpers", "fp32_chain.c")
+    lib = str(tmp_path_factory.mktemp("fp32") / "libfp32_chain.so")
+    subprocess.run(["gcc", "-O1", "-frounding-math", "-ffp-contract=off", "-fPIC", "-shared", src, "-o", lib, "-lm"],
+                   check=True)
+    dll = ctypes.CDLL(lib)
+    dll.fp32_chain.restype = ctypes.c_float
+    dll.fp32_chain.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float), ctypes.c_int64,
+                               ctypes.c_int]
+
+    def run(x, w, toward_zero):
+        x = np.ascontiguousarray(x, np.float32)
+        w = np.ascontiguousarray(w, np.float32)
+        return float(dll.fp32_chain(x.ctypes.data_as(ctypes.POINTER(ctypes.c_float)),
+                                    w.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), len(x), int(toward_zero)))
+    return run
+
+
+@pytest.mark.parametrize("K", [1, 7, 64, 577, 3000])
+def test_wide_accumulator_is_ieee_binary32_summation(fp32_chain, K):
+    # (M23, E8, b=127): R_UF = 2^-127 and R_OF > 2^128 cannot be reached from E4M3 products, so
+    # FMAq is one correctly rounded binary32 addition per step (Eq. 4 with Q = binary32 rounding).
+    for trial in range(4):
+        x = synth.random_codes((K,), 100 + trial).numpy()
+        w = synth.random_codes((K,), 200 + trial).numpy()
+        xf, wf = _decode_f32(x), _decode_f32(w)
+        s = np.float32(0)
+        for a, b in zip(xf, wf):
+            s = np.float32(s + np.float32(a * b))
+        assert orc.dot(WIDE_NEAREST, WIDE_NEAREST, SEQ, 16, x, w) == float(s)
+        assert fp32_chain(xf, wf, False) == float(s)
+        assert orc.dot(WIDE_FLOOR, WIDE_FLOOR, SEQ, 16, x, w) == fp32_chain(xf, wf, True)
+
+
+def test_chunk_extremes_equal_sequential():
+    prod, acc = (7, 4, -2, 0, 1), (7, 4, -4, 0, 1)
+    for K in (1, 5, 16, 17, 100):
+        x = synth.random_codes((K,), 31 + K).numpy()
+        w = synth.random_codes((K,), 41 + K).numpy()
+        seq = orc.dot(prod, acc, SEQ, 16, x, w)
+        assert orc.dot(prod, acc, CHK, K, x, w) == seq          # one chunk: second level adds 0
+        assert orc.dot(prod, acc, CHK, K + 5, x, w) == seq
+        # chunks of one compute Q_acc(Q_acc(P) + T): the same as sequential whenever Q_acc leaves a
+        # lone product unchanged, e.g. when both quantisers share one format
+        same = (7, 4, -2, 0, 1)
+        assert orc.dot(same, same, CHK, 1, x, w) == orc.dot(same, same, SEQ, 16, x, w)
+
+
+def test_order_is_observable():
+    # Sec. 3 / App. D: accumulation order changes the result because of swamping
+    prod, acc = (7, 4, -2, 0, 1), (7, 4, -4, 0, 1)
+    differ = 0
+    for t in range(20):
+        a, _, b, _ = synth.gemm_case(1, 1, 576, 900 + t)
+        differ += orc.dot(prod, acc, SEQ, 16, a[0].numpy(), b[0].numpy()) != orc.dot(prod, acc, CHK, 16, a[0].numpy(),
+                                                                                       b[0].numpy())
+    assert differ > 0
+
+
+@pytest.mark.parametrize("order,chunk", [(SEQ, 16), (CHK, 16), (CHK, 5)])
+def test_exact_when_all_partial_sums_are_representable(order, chunk):
+    # small integers, 10-bit mantissa, wide range: nothing is ever rounded, so the result is the integer dot product
+    prod, acc = (10, 6, 20, 0, 1), (10, 6, 20, 0, 1)
+    for t in range(10):
+        x = synth.small_integer_codes((40,), 300 + t, max_abs=5)
+        w = synth.small_integer_codes((40,), 400 + t, max_abs=5)
+        want = int(np.dot(_decode_f32(x.numpy()).astype(np.int64), _decode_f32(w.numpy()).astype(np.int64)))
+        assert abs(want) < 1024
+        assert orc.dot(prod, acc, order, chunk, x.numpy(), w.numpy()) == float(want)
+
+
+def test_zero_products_leave_the_sum_unchanged():
+    # FMAq(0, w, S) = Q_acc(S) = S: the fact that makes padded convolution taps and K padding harmless
+    prod, acc = (7, 4, -2, 0, 1), (7, 4, -4, 0, 1)
+    x = synth.random_codes((64,), 1).numpy()
+    w = synth.random_codes((64,), 2).numpy()
+    base = orc.dot(prod, acc, SEQ, 16, x, w)
+    xz = np.concatenate([x, np.zeros(9, np.uint8), np.full(3, 0x80, np.uint8)])
+    wz = np.concatenate([w, synth.random_codes((12,), 3).numpy()])
+    assert orc.dot(prod, acc, SEQ, 16, xz, wz) == base
+
+
+FORMAT_PAIRS = [((7, 4, -2), (7, 4, -4)), ((7, 4, 12), (7, 4, 10)), ((4, 4, -2), (4, 4, -4)), ((5, 5, 14), (5, 5, 12)),
+                ((10, 6, 46), (10, 6, 44)), ((4, 3, 5), (4, 3, 5)), ((3, 4, 2), (9, 5, 9))]
+
+
+@pytest.mark.parametrize("rounding", [0, 1])
+def test_brute_force_all_pairs_k1(rounding):
+    # every finite E4M3 pair through one FMAq from S = 0, against the exact-rational coding
+    codes = FINITE
+    for pf, af in FORMAT_PAIRS[:4]:
+        prod, acc = pf + (rounding, 1), af + (rounding, 1)
+        A = codes[:, None]
+        out = orc.gemm(A, A, 1.0, 1.0, None, prod, acc, SEQ, 16)     # out[i][j] = FMAq(c_i, c_j, 0)
+        vals = [ex.decode_e4m3(int(c)) for c in codes]
+        for i in range(0, len(codes)):
+            for j in range(i % 3, len(codes), 3):                    # a third of the pairs exactly checked
+                want = ex.quantise(acc, ex.quantise(prod, vals[i] * vals[j]))
+                assert Fraction(float(out[i, j])) == want, (pf, af, i, j)
+
+
+@pytest.mark.parametrize("rounding", [0, 1])
+@pytest.mark.parametrize("K", [2, 3, 4, 33])
+def test_sampled_chains_against_exact_rationals(K, rounding):
+    for fi, (pf, af) in enumerate(FORMAT_PAIRS):
+        for flags in (1, 0):
+            prod, acc = pf + (rounding, flags), af + (rounding, flags)
+            for t in range(25 if K <= 4 else 6):
+                x = synth.random_codes((K,), 5000 + 97 * fi + t).numpy()
+                w = synth.random_codes((K,), 6000 + 89 * fi + t).numpy()
+                for order, chunk in ((SEQ, 16), (CHK, 16), (CHK, 2)):
+                    got = orc.dot(prod, acc, order, chunk, x, w)
+                    assert Fraction(got) == ex.dot(prod, acc, order, chunk, x, w), (prod, acc, order, chunk, t)
+
+
+def test_planted_mistakes_are_caught_by_the_pins():
+    """Each plausible slip, applied to the exact-rational coding, must break a hand-worked value."""
+    x = [ex.decode_e4m3(0x48)] * 5
+    prod, acc = (7, 4, 12, 0, 1), (7, 4, 10, 0, 1)
+
+    def chain(q_prod, q_acc, n=5):
+        s = Fraction(0)
+        for a in x[:n]:
+            s = q_acc(q_prod(a * a) + s)
+        return s
+    good = chain(lambda v: ex.quantise(prod, v), lambda v: ex.quantise(acc, v))
+    assert good == Fraction(63.75)
+    # dropped Q_prod
+    assert chain(lambda v: v, lambda v: ex.quantise(acc, v), 3) != Fraction(47.75)
+    # Q_acc applied only at the end of the sum instead of after every addition
+    s3 = sum(ex.quantise(prod, a * a) for a in x[:3])
+    s4 = ex.quantise(acc, s3 + ex.quantise(prod, x[3] * x[3]))
+    assert s4 != Fraction(63.5)          # 47.8125 + 15.9375 = 63.75 exactly; per-step rounding gives 63.5
+    # biases swapped
+    assert chain(lambda v: ex.quantise(acc, v), lambda v: ex.quantise(prod, v), 2) != Fraction(31.875)
+    # nearest instead of floor
+    assert chain(lambda v: ex.quantise(prod, v), lambda v: ex.quantise((7, 4, 10, 1, 1), v), 4) != Fraction(63.5)
+    # last product dropped (the S_{N-1} misprint of Eq. 8-9)
+    assert chain(lambda v: ex.quantise(prod, v), lambda v: ex.quantise(acc, v), 4) != good
