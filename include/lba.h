@@ -1,0 +1,149 @@
+/* liblba: GEMM and 2-D convolution with a low bit-width floating-point accumulator (LBA)
+ * on NVIDIA B200 (sm_100a).  C ABI; no CUDA or C++ types appear in any signature.
+ *
+ * What every call computes, for each output scalar (paper: "Towards Cheaper Inference in
+ * Deep Networks with Lower Bit-Width Accumulators"):
+ *
+ *     y = sum_i x_i * w_i                                             Eq. 3
+ *
+ * with the fused multiply-add replaced by
+ *
+ *     FMAq(x, w, s) = Q_acc( Q_prod(x * w) + s )                       Eq. 4
+ *
+ * where Q is the floating-point quantiser Q^FLOAT_{M,E,b} of Eq. 2 (saturate at
+ * R_OF = 2^(2^E-b-1) * (2 - 2^-M), flush to zero below R_UF = 2^-b, no subnormals, mantissa
+ * cut to M bits).  The product and the sum inside Eq. 4 are exact; each is rounded once.
+ * Inputs are OCP FP8 E4M3 bytes; arithmetic runs on their decoded values ("code domain");
+ * real-valued scales are applied to the finished sum in binary32, outside the FMAq unit
+ * (Fig. 1, left: W/A quantisation is software, Q_prod/Q_acc are the simulated hardware).
+ *
+ * Accumulation order (it changes the result, App. D):
+ *   LBA_ORDER_SEQUENTIAL  S_0 = 0, S_{i+1} = FMAq(x_i, w_i, S_i), y = S_K       Eq. 8-9
+ *   LBA_ORDER_CHUNKED     two hierarchies (Sec. 3, Fig. 1 right, App. D): each run of `chunk`
+ *                         consecutive products is accumulated sequentially from 0; the chunk
+ *                         sums are then added in chunk order, from 0, with Q_acc after every
+ *                         addition (no Q_prod at that level).  The paper uses chunk = 16.
+ *                         The last chunk may be short.
+ *
+ * All device pointers must belong to the current CUDA device.  The library allocates no
+ * memory, keeps no state between calls except the last CUDA error code, and never
+ * synchronises: work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default
+ * stream).  Format structs are read on the host during the call.
+ *
+ * Preconditions that are not checked on the device: no input byte is an E4M3 NaN code
+ * (0x7F, 0xFF; use lba_count_nan_codes to check), scales are finite and > 0.  Every zero
+ * produced by the chain is +0.
+ */
+#ifndef LBA_H_
+#define LBA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Q^FLOAT_{M,E,b} of Eq. 2. */
+typedef struct {
+  int32_t man_bits; /* M, 1..23                                                             */
+  int32_t exp_bits; /* E, 1..8: binades [-b, 2^E-b-1], none reserved                        */
+  int32_t bias;     /* b, -96..192                                                          */
+  int32_t rounding; /* LBA_ROUND_FLOOR (the paper's, Sec. 3) or LBA_ROUND_NEAREST_EVEN      */
+  int32_t flags;    /* bit0 LBA_FLAG_UNDERFLOW: 1 = flush |x| < R_UF to 0 (Eq. 2);
+                       0 = "excluding underflow" (first fine-tuning stage, Sec. 3)          */
+} lba_fmt;
+
+enum { LBA_ROUND_FLOOR = 0, LBA_ROUND_NEAREST_EVEN = 1 };
+enum { LBA_FLAG_UNDERFLOW = 1 };
+enum { LBA_ORDER_SEQUENTIAL = 0, LBA_ORDER_CHUNKED = 1 };
+
+enum {
+  LBA_OK = 0,
+  LBA_ERR_NULL = -1,      /* a required pointer is NULL                                      */
+  LBA_ERR_SHAPE = -2,     /* a negative size, an empty convolution output, sizes beyond int32
+                             where the kernel indexes with int32                             */
+  LBA_ERR_FORMAT = -3,    /* M/E/b/rounding out of range, or a format whose reachable values
+                             cannot be carried exactly in binary32 registers                 */
+  LBA_ERR_ORDER = -4,     /* unknown order, or chunk < 1 in chunked order                    */
+  LBA_ERR_SCALE_LEN = -5, /* a scale length that is neither 1 nor the matching dimension     */
+  LBA_ERR_CUDA = -6,      /* a CUDA call failed; see lba_last_cuda_error                     */
+  LBA_ERR_WORKSPACE = -7  /* host-buffer entry points: workspace NULL, too small, misaligned */
+};
+
+/* GEMM  out[m][n] = epilogue( dot(A[m][:], B[n][:]) ), i.e. Y = X W^T with x_i = X_mi,
+ * w_i = W_ni (App. A).
+ *   A        device, [M][K] E4M3 bytes, K contiguous
+ *   B        device, [N][K] E4M3 bytes, K contiguous
+ *   scale_a  device, 1 value (per tensor) or M values (per row); scale_a_len says which
+ *   scale_b  device, 1 value or N values (per output channel)
+ *   bias     device, N values, or NULL
+ *   out      device, [M][N] binary32, row-major; out = fl(fl(y*scale_a)*scale_b) (+ bias)
+ * 16-byte aligned A and B with K a multiple of 16 take the vector-load path; anything else
+ * is accepted and takes a slower byte-wise loader with identical results.
+ * M, N or K equal to 0 are legal (K = 0 gives y = 0).  Returns LBA_OK or a negative code;
+ * on error nothing is enqueued. */
+int lba_gemm(const uint8_t* A, const uint8_t* B, const float* scale_a, int scale_a_len, const float* scale_b,
+             int scale_b_len, const float* bias, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt,
+             const lba_fmt* acc_fmt, int order, int chunk, float* out, void* stream);
+
+/* Convolution as an implicit GEMM (Eq. 3 with m = (b, oh, ow), n = c_out and k walking
+ * (kh, kw, c_in), c_in fastest).  Padded taps are the value 0 and still count toward the
+ * chunk position.  Dilation 1, groups 1.
+ *   x        device, [B][H][W][C_in] E4M3 bytes (NHWC)
+ *   w        device, [C_out][KH][KW][C_in] E4M3 bytes
+ *   scale_x  device, 1 value or B*H_out*W_out values; scale_w: 1 or C_out values
+ *   bias     device, C_out values, or NULL
+ *   out      device, [B][H_out][W_out][C_out] binary32,
+ *            H_out = (H + 2*pad_h - KH)/stride_h + 1, likewise W_out
+ * C_in a multiple of 16 with 16-byte aligned x and w takes the vector-load path. */
+int lba_conv2d(const uint8_t* x, const uint8_t* w, const float* scale_x, int scale_x_len, const float* scale_w,
+               int scale_w_len, const float* bias, int B, int H, int W, int C_in, int C_out, int KH, int KW,
+               int stride_h, int stride_w, int pad_h, int pad_w, const lba_fmt* prod_fmt, const lba_fmt* acc_fmt,
+               int order, int chunk, float* out, void* stream);
+
+/* The same two operations on HOST buffers (pinned memory recommended): inputs are copied to
+ * the caller's device workspace, the kernel runs, and `out` (host) receives the result; all
+ * of it is enqueued on `stream`, so the caller synchronises the stream before reading `out`.
+ * `workspace` is device memory, 256-byte aligned, of at least lba_*_host_workspace_bytes(...)
+ * bytes; the library does not allocate. */
+size_t lba_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int scale_a_len, int scale_b_len,
+                                     int has_bias);
+int lba_gemm_host(const uint8_t* A, const uint8_t* B, const float* scale_a, int scale_a_len, const float* scale_b,
+                  int scale_b_len, const float* bias, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt,
+                  const lba_fmt* acc_fmt, int order, int chunk, float* out, void* workspace,
+                  size_t workspace_bytes, void* stream);
+size_t lba_conv2d_host_workspace_bytes(int B, int H, int W, int C_in, int C_out, int KH, int KW, int stride_h,
+                                       int stride_w, int pad_h, int pad_w, int scale_x_len, int scale_w_len,
+                                       int has_bias);
+int lba_conv2d_host(const uint8_t* x, const uint8_t* w, const float* scale_x, int scale_x_len,
+                    const float* scale_w, int scale_w_len, const float* bias, int B, int H, int W, int C_in,
+                    int C_out, int KH, int KW, int stride_h, int stride_w, int pad_h, int pad_w,
+                    const lba_fmt* prod_fmt, const lba_fmt* acc_fmt, int order, int chunk, float* out,
+                    void* workspace, size_t workspace_bytes, void* stream);
+
+/* Debug helper for the NaN-code precondition: adds to *count (device, uint64, caller zeroes
+ * it) the number of bytes among codes[0..n) equal to 0x7F or 0xFF. */
+int lba_count_nan_codes(const uint8_t* codes, int64_t n, unsigned long long* count, void* stream);
+
+/* Which kernel variant a call with these arguments would run, as text, e.g.
+ * "tile=128x128x16 micro=8x8 q=floor_fast order=chunk_slab load=gemm_vec grid=64x64".
+ * is_conv selects the loader family; for a convolution pass M = B*H_out*W_out, N = C_out,
+ * K = KH*KW*C_in and vec_ok = (C_in % 16 == 0 and pointers aligned).  Returns LBA_OK or the
+ * error the real call would return; buf may be NULL. */
+int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, const lba_fmt* acc_fmt, int order,
+                      int chunk, int is_conv, int vec_ok, char* buf, size_t buf_len);
+
+/* Testing and tuning hook: force the CTA tile (0 = 128x128, 1 = 128x64, 2 = 64x64, 3 = 32x32
+ * outputs; -1 = automatic choice, the default).  Process-wide; results never depend on the tile,
+ * only speed does.  Returns LBA_OK, or LBA_ERR_SHAPE for an unknown tile. */
+int lba_set_tile_override(int tile);
+
+const char* lba_status_string(int status);
+int lba_last_cuda_error(void); /* cudaError_t of the most recent failed CUDA call in this thread, else 0 */
+int lba_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LBA_H_ */

@@ -1,0 +1,456 @@
+// C ABI of liblba: argument checks, the per-call arithmetic plan, tile choice and dispatch.
+// The definitions of the operations are in include/lba.h; the kernel is in lba_kernel.cuh.
+#include <cfloat>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "../../include/lba.h"
+#include "lba_kernel.cuh"
+
+namespace lba {
+
+// one definition per (QM, ORD), in the lba_fam_*.cu translation units
+#define LBA_DECL(QM, ORD) template <> cudaError_t launch_family<QM, ORD>(int, int, const Problem&, cudaStream_t);
+LBA_DECL(QM_FLOOR_FAST, ORD_SEQ) LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK_SLAB) LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK_ANY)
+LBA_DECL(QM_FLOOR_FULL, ORD_SEQ) LBA_DECL(QM_FLOOR_FULL, ORD_CHUNK_SLAB) LBA_DECL(QM_FLOOR_FULL, ORD_CHUNK_ANY)
+LBA_DECL(QM_RNE_FULL, ORD_SEQ) LBA_DECL(QM_RNE_FULL, ORD_CHUNK_SLAB) LBA_DECL(QM_RNE_FULL, ORD_CHUNK_ANY)
+LBA_DECL(QM_RNE_WIDE, ORD_SEQ) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_SLAB) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_ANY)
+#undef LBA_DECL
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+int g_tile_override = -1;
+
+int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return LBA_ERR_CUDA;
+}
+
+const LaunchFn kLaunch[QM_COUNT][ORD_COUNT] = {
+    {launch_family<QM_FLOOR_FAST, ORD_SEQ>, launch_family<QM_FLOOR_FAST, ORD_CHUNK_SLAB>,
+     launch_family<QM_FLOOR_FAST, ORD_CHUNK_ANY>},
+    {launch_family<QM_FLOOR_FULL, ORD_SEQ>, launch_family<QM_FLOOR_FULL, ORD_CHUNK_SLAB>,
+     launch_family<QM_FLOOR_FULL, ORD_CHUNK_ANY>},
+    {launch_family<QM_RNE_FULL, ORD_SEQ>, launch_family<QM_RNE_FULL, ORD_CHUNK_SLAB>,
+     launch_family<QM_RNE_FULL, ORD_CHUNK_ANY>},
+    {launch_family<QM_RNE_WIDE, ORD_SEQ>, launch_family<QM_RNE_WIDE, ORD_CHUNK_SLAB>,
+     launch_family<QM_RNE_WIDE, ORD_CHUNK_ANY>},
+};
+
+const char* const kQmName[QM_COUNT] = {"floor_fast", "floor_full", "rne_full", "rne_wide"};
+const char* const kOrdName[ORD_COUNT] = {"seq", "chunk_slab", "chunk_any"};
+const char* const kLdName[LD_COUNT] = {"gemm_vec", "conv_vec", "any"};
+
+// Largest |x*w| of two E4M3 values and the grid every product lies on.
+constexpr double kMaxProduct = 448.0 * 448.0;  // 200704
+constexpr int kMinProductExp = -18;            // every product, hence every sum, is a multiple of 2^-18
+
+struct Plan {
+  int qm, ord;
+  float dec_a, dec_b, c, un1, un2;
+  QConst qp, qa;
+  int chunk_slabs, chunk;
+};
+
+bool fmt_ok(const lba_fmt* f) {
+  return f->man_bits >= 1 && f->man_bits <= 23 && f->exp_bits >= 1 && f->exp_bits <= 8 && f->bias >= -96 &&
+         f->bias <= 192 && (f->rounding == LBA_ROUND_FLOOR || f->rounding == LBA_ROUND_NEAREST_EVEN);
+}
+
+double r_of(const lba_fmt* f) {  // Eq. 2; exact in double for the admitted M, E, b
+  return std::ldexp(2.0 - std::ldexp(1.0, -f->man_bits), (1 << f->exp_bits) - f->bias - 1);
+}
+
+void fill_qconst(QConst* q, int M, float sat) {
+  const int sh = 23 - M;
+  q->mask = sh == 0 ? 0xFFFFFFFFu : ~((1u << sh) - 1u);
+  q->rne_shift = sh;
+  q->rne_add = sh == 0 ? 0u : ((1u << (sh - 1)) - 1u);
+  q->rne_lsb = sh == 0 ? 0u : 1u;
+  q->sat = sat;
+}
+
+// Work out, on the host, how the two formats are carried in binary32 registers and which of the
+// branches of Eq. 2 can be reached at all from E4M3 inputs; refuse what cannot be carried exactly.
+int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_t K, Plan* pl) {
+  if (!pf || !af) return LBA_ERR_NULL;
+  if (!fmt_ok(pf) || !fmt_ok(af)) return LBA_ERR_FORMAT;
+  if (pf->rounding != af->rounding) return LBA_ERR_FORMAT;  // one rounding rule per FMAq unit
+  if (order != LBA_ORDER_SEQUENTIAL && order != LBA_ORDER_CHUNKED) return LBA_ERR_ORDER;
+  if (order == LBA_ORDER_CHUNKED && chunk < 1) return LBA_ERR_ORDER;
+  const bool nearest = af->rounding == LBA_ROUND_NEAREST_EVEN;
+
+  // ---- Q_prod
+  const bool p_flush = (pf->flags & LBA_FLAG_UNDERFLOW) && pf->bias < -kMinProductExp;  // R_UF_prod > 2^-18
+  const int kp = p_flush ? pf->bias - 126 : -108;  // carrier = value * 2^kp; 2^-18 * 2^-108 is still normal
+  const double p_rof = r_of(pf);
+  // nearest-even can carry a value in the last half step below R_OF past it, so reachability
+  // is judged with that margin; floor never increases a magnitude
+  const bool p_sat = p_rof <= kMaxProduct * (nearest ? 1.0 + std::ldexp(1.0, -pf->man_bits - 1) : 1.0);
+  const bool p_round = pf->man_bits < 7;  // an E4M3 product has at most 8 significant bits
+  const int p_emax = (1 << pf->exp_bits) - pf->bias - 1;
+  float p_sat_carrier = FLT_MAX;
+  if (p_sat) {
+    if (p_emax + kp < -126 || p_emax + kp > 127) return LBA_ERR_FORMAT;
+    p_sat_carrier = (float)std::ldexp(p_rof, kp);
+  }
+  // ---- Q_acc
+  const bool a_flush = (af->flags & LBA_FLAG_UNDERFLOW) && af->bias < -kMinProductExp;
+  const int ka = a_flush ? af->bias - 126 : -108;
+  const double a_rof = r_of(af);
+  const double max_term = p_sat ? p_rof : kMaxProduct;
+  // |S_i| <= i * max_term under floor; under nearest-even each step may add half a grid step
+  const double growth = nearest ? std::exp(std::fmin((double)(K > 0 ? K : 1) * std::ldexp(1.0, -af->man_bits - 1), 80.0)) : 1.0;
+  const double max_sum = (double)(K > 0 ? K : 1) * max_term * growth;
+  const bool a_sat = a_rof <= max_sum;
+  const int a_emax = (1 << af->exp_bits) - af->bias - 1;
+  float a_sat_carrier = FLT_MAX;
+  if (a_sat) {
+    if (a_emax + ka < -126 || a_emax + ka > 127) return LBA_ERR_FORMAT;
+    a_sat_carrier = (float)std::ldexp(a_rof, ka);
+  } else if (std::ldexp(max_sum, ka) >= std::ldexp(1.0, 127)) {
+    return LBA_ERR_FORMAT;
+  }
+  if (ka - kp < -126 || ka - kp > 126) return LBA_ERR_FORMAT;
+  // the finished sum must be a normal binary32 number in the real domain: reachable magnitudes
+  // lie in [2^-18, min(R_OF_acc, max_sum)]
+  if ((a_sat ? a_rof : max_sum) >= std::ldexp(1.0, 128)) return LBA_ERR_FORMAT;
+
+  // ---- quantiser mode
+  if (!nearest) {
+    pl->qm = (p_round || p_sat) ? QM_FLOOR_FULL : QM_FLOOR_FAST;
+  } else if (af->man_bits == 23) {
+    // a 24-bit accumulator is one IEEE addition, provided nothing else of Eq. 2 can happen
+    if (p_flush || a_flush || p_sat || a_sat || p_round) return LBA_ERR_FORMAT;
+    pl->qm = QM_RNE_WIDE;
+  } else if (af->man_bits == 22) {
+    return LBA_ERR_FORMAT;  // round-to-odd needs two spare bits below the kept mantissa
+  } else {
+    pl->qm = QM_RNE_FULL;
+  }
+  fill_qconst(&pl->qp, pf->man_bits, p_sat_carrier);
+  fill_qconst(&pl->qa, af->man_bits, a_sat_carrier);
+
+  const int sx = (kp >= 0) ? kp / 2 : -((-kp + 1) / 2);  // floor(kp / 2)
+  const int sw = kp - sx;
+  pl->dec_a = (float)std::ldexp(1.0, 120 + sx);
+  pl->dec_b = (float)std::ldexp(1.0, 120 + sw);
+  pl->c = (float)std::ldexp(1.0, ka - kp);
+  const int u1 = (-ka) / 2, u2 = (-ka) - u1;
+  pl->un1 = (float)std::ldexp(1.0, u1);
+  pl->un2 = (float)std::ldexp(1.0, u2);
+
+  // ---- order mode
+  pl->chunk = chunk;
+  pl->chunk_slabs = 0;
+  if (order == LBA_ORDER_SEQUENTIAL || (int64_t)chunk >= K) {
+    pl->ord = ORD_SEQ;  // a single chunk: the second hierarchy adds it to 0, which changes nothing
+  } else if (chunk % BK == 0) {
+    pl->ord = ORD_CHUNK_SLAB;
+    pl->chunk_slabs = chunk / BK;
+  } else {
+    pl->ord = ORD_CHUNK_ANY;
+  }
+  return LBA_OK;
+}
+
+// Tile choice: the largest tile that still gives every SM work; smaller tiles cost more loads and
+// decodes per MAC, larger ones leave SMs idle on small problems.
+int choose_tile(int64_t M, int64_t N, int ord) {
+  if (g_tile_override >= 0) return g_tile_override;
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
+  }
+  // CTAs resident per SM (register-limited) and relative per-MAC efficiency of each tile
+  const int resident[TILE_COUNT] = {1, ord == ORD_SEQ ? 2 : 2, 3, 8};
+  const double eff[TILE_COUNT] = {1.00, 0.97, 0.92, 0.80};
+  int best = 0;
+  double best_cost = 1e300;
+  for (int t = 0; t < TILE_COUNT; ++t) {
+    const TileInfo ti = tile_info(t);
+    const double ctas = (double)((M + ti.bm - 1) / ti.bm) * (double)((N + ti.bn - 1) / ti.bn);
+    const double slots = (double)sms * resident[t];
+    const double waves = std::ceil(ctas / slots);
+    // time ~ waves * (work of the CTAs sharing an SM) / efficiency
+    const double cost = waves * resident[t] * ti.bm * ti.bn / eff[t];
+    if (cost < best_cost) {
+      best_cost = cost;
+      best = t;
+    }
+  }
+  return best;
+}
+
+int fill_scales(Problem* p, const float* sa, int sa_len, const float* sb, int sb_len, const float* bias) {
+  if (!sa || !sb) return LBA_ERR_NULL;
+  if (!(sa_len == 1 || (int64_t)sa_len == p->M) || !(sb_len == 1 || (int64_t)sb_len == p->N))
+    return LBA_ERR_SCALE_LEN;
+  p->sa = sa;
+  p->sb = sb;
+  p->bias = bias;
+  p->sa_per_row = sa_len != 1 ? 1 : 0;
+  p->sb_per_col = sb_len != 1 ? 1 : 0;
+  return LBA_OK;
+}
+
+void apply_plan(Problem* p, const Plan& pl) {
+  p->dec_a = pl.dec_a;
+  p->dec_b = pl.dec_b;
+  p->c = pl.c;
+  p->un1 = pl.un1;
+  p->un2 = pl.un2;
+  p->qp = pl.qp;
+  p->qa = pl.qa;
+  p->chunk_slabs = pl.chunk_slabs;
+  p->chunk = pl.chunk;
+}
+
+bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0; }
+
+int run(const Problem& p, const Plan& pl, int load, cudaStream_t stream) {
+  if (p.M == 0 || p.N == 0) return LBA_OK;
+  const int tile = choose_tile(p.M, p.N, pl.ord);
+  const TileInfo ti = tile_info(tile);
+  if ((p.N + ti.bn - 1) / ti.bn > 65535 || (p.M + ti.bm - 1) / ti.bm > 2147483647LL) return LBA_ERR_SHAPE;
+  const cudaError_t e = kLaunch[pl.qm][pl.ord](tile, load, p, stream);
+  return e == cudaSuccess ? LBA_OK : cuda_fail(e);
+}
+
+struct ConvGeom {
+  int Hout, Wout;
+  int64_t M, K;
+};
+
+int conv_geom(int B, int H, int W, int C_in, int C_out, int KH, int KW, int sh, int sw, int ph, int pw,
+              ConvGeom* g) {
+  if (B < 1 || H < 1 || W < 1 || C_in < 1 || C_out < 1 || KH < 1 || KW < 1 || sh < 1 || sw < 1 || ph < 0 || pw < 0)
+    return LBA_ERR_SHAPE;
+  if ((int64_t)H + 2 * (int64_t)ph < KH || (int64_t)W + 2 * (int64_t)pw < KW) return LBA_ERR_SHAPE;
+  g->Hout = (H + 2 * ph - KH) / sh + 1;
+  g->Wout = (W + 2 * pw - KW) / sw + 1;
+  if (g->Hout < 1 || g->Wout < 1) return LBA_ERR_SHAPE;
+  g->M = (int64_t)B * g->Hout * g->Wout;
+  g->K = (int64_t)KH * KW * C_in;
+  if (g->K > 2147483647LL || (int64_t)H * W * C_in > 2147483647LL) return LBA_ERR_SHAPE;
+  return LBA_OK;
+}
+
+__global__ void count_nan_codes_kernel(const uint8_t* codes, int64_t n, unsigned long long* count) {
+  unsigned long long local = 0;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    local += (codes[i] & 0x7F) == 0x7F;
+  if (local) atomicAdd(count, local);
+}
+
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+}  // namespace lba
+
+using namespace lba;
+
+extern "C" {
+
+int lba_version(void) { return 1; }
+
+int lba_last_cuda_error(void) { return g_last_cuda_error; }
+
+int lba_set_tile_override(int tile) {
+  if (tile < -1 || tile >= TILE_COUNT) return LBA_ERR_SHAPE;
+  g_tile_override = tile;
+  return LBA_OK;
+}
+
+const char* lba_status_string(int status) {
+  switch (status) {
+    case LBA_OK: return "ok";
+    case LBA_ERR_NULL: return "a required pointer is NULL";
+    case LBA_ERR_SHAPE: return "bad shape";
+    case LBA_ERR_FORMAT: return "format out of range or not exactly representable in the binary32 carrier";
+    case LBA_ERR_ORDER: return "unknown accumulation order or chunk < 1";
+    case LBA_ERR_SCALE_LEN: return "scale length must be 1 or the matching dimension";
+    case LBA_ERR_CUDA: return "a CUDA call failed (see lba_last_cuda_error)";
+    case LBA_ERR_WORKSPACE: return "workspace missing, too small or misaligned";
+    default: return "unknown status";
+  }
+}
+
+int lba_gemm(const uint8_t* A, const uint8_t* B, const float* scale_a, int scale_a_len, const float* scale_b,
+             int scale_b_len, const float* bias, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt,
+             const lba_fmt* acc_fmt, int order, int chunk, float* out, void* stream) {
+  if (M < 0 || N < 0 || K < 0 || K > 2147483647LL) return LBA_ERR_SHAPE;
+  Plan pl;
+  int st = make_plan(prod_fmt, acc_fmt, order, chunk, K, &pl);
+  if (st != LBA_OK) return st;
+  Problem p;
+  std::memset(&p, 0, sizeof(p));
+  p.M = M;
+  p.N = N;
+  p.K = K;
+  if ((st = fill_scales(&p, scale_a, scale_a_len, scale_b, scale_b_len, bias)) != LBA_OK) return st;
+  if (M > 0 && N > 0 && !out) return LBA_ERR_NULL;
+  if (K > 0 && ((M > 0 && !A) || (N > 0 && !B))) return LBA_ERR_NULL;
+  p.A = A;
+  p.B = B;
+  p.out = out;
+  apply_plan(&p, pl);
+  const bool vec = K % BK == 0 && aligned16(A) && aligned16(B);
+  return run(p, pl, vec ? LD_GEMM_VEC : LD_ANY, (cudaStream_t)stream);
+}
+
+int lba_conv2d(const uint8_t* x, const uint8_t* w, const float* scale_x, int scale_x_len, const float* scale_w,
+               int scale_w_len, const float* bias, int B, int H, int W, int C_in, int C_out, int KH, int KW,
+               int stride_h, int stride_w, int pad_h, int pad_w, const lba_fmt* prod_fmt, const lba_fmt* acc_fmt,
+               int order, int chunk, float* out, void* stream) {
+  ConvGeom g;
+  int st = conv_geom(B, H, W, C_in, C_out, KH, KW, stride_h, stride_w, pad_h, pad_w, &g);
+  if (st != LBA_OK) return st;
+  Plan pl;
+  if ((st = make_plan(prod_fmt, acc_fmt, order, chunk, g.K, &pl)) != LBA_OK) return st;
+  if (!x || !w || !out) return LBA_ERR_NULL;
+  Problem p;
+  std::memset(&p, 0, sizeof(p));
+  p.M = g.M;
+  p.N = C_out;
+  p.K = g.K;
+  if ((st = fill_scales(&p, scale_x, scale_x_len, scale_w, scale_w_len, bias)) != LBA_OK) return st;
+  p.A = x;
+  p.B = w;
+  p.out = out;
+  p.is_conv = 1;
+  p.H = H; p.W = W; p.Cin = C_in; p.KH = KH; p.KW = KW;
+  p.sh = stride_h; p.sw = stride_w; p.ph = pad_h; p.pw = pad_w;
+  p.Hout = g.Hout; p.Wout = g.Wout;
+  apply_plan(&p, pl);
+  const bool vec = C_in % BK == 0 && aligned16(x) && aligned16(w);
+  return run(p, pl, vec ? LD_CONV_VEC : LD_ANY, (cudaStream_t)stream);
+}
+
+size_t lba_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int scale_a_len, int scale_b_len,
+                                     int has_bias) {
+  if (M < 0 || N < 0 || K < 0 || scale_a_len < 0 || scale_b_len < 0) return 0;
+  size_t b = 0;
+  b += round_up((size_t)M * K, 256) + round_up((size_t)N * K, 256);
+  b += round_up((size_t)scale_a_len * 4, 256) + round_up((size_t)scale_b_len * 4, 256);
+  if (has_bias) b += round_up((size_t)N * 4, 256);
+  b += round_up((size_t)M * N * 4, 256);
+  return b;
+}
+
+int lba_gemm_host(const uint8_t* A, const uint8_t* B, const float* scale_a, int scale_a_len, const float* scale_b,
+                  int scale_b_len, const float* bias, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt,
+                  const lba_fmt* acc_fmt, int order, int chunk, float* out, void* workspace,
+                  size_t workspace_bytes, void* stream) {
+  if (M < 0 || N < 0 || K < 0) return LBA_ERR_SHAPE;
+  if (!scale_a || !scale_b) return LBA_ERR_NULL;
+  if (!(scale_a_len == 1 || scale_a_len == M) || !(scale_b_len == 1 || scale_b_len == N)) return LBA_ERR_SCALE_LEN;
+  Plan pl;
+  int st = make_plan(prod_fmt, acc_fmt, order, chunk, K, &pl);  // reject bad formats before any copy
+  if (st != LBA_OK) return st;
+  const size_t need = lba_gemm_host_workspace_bytes(M, N, K, scale_a_len, scale_b_len, bias != nullptr);
+  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255)) return LBA_ERR_WORKSPACE;
+  if ((M * K > 0 && !A) || (N * K > 0 && !B) || (M * N > 0 && !out)) return LBA_ERR_NULL;
+  cudaStream_t s = (cudaStream_t)stream;
+  uint8_t* w = (uint8_t*)workspace;
+  uint8_t* dA = w; w += round_up((size_t)M * K, 256);
+  uint8_t* dB = w; w += round_up((size_t)N * K, 256);
+  float* dsa = (float*)w; w += round_up((size_t)scale_a_len * 4, 256);
+  float* dsb = (float*)w; w += round_up((size_t)scale_b_len * 4, 256);
+  float* dbias = nullptr;
+  if (bias) { dbias = (float*)w; w += round_up((size_t)N * 4, 256); }
+  float* dout = (float*)w;
+  cudaError_t e;
+  if (M * K > 0 && (e = cudaMemcpyAsync(dA, A, (size_t)M * K, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+  if (N * K > 0 && (e = cudaMemcpyAsync(dB, B, (size_t)N * K, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(dsa, scale_a, (size_t)scale_a_len * 4, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(dsb, scale_b, (size_t)scale_b_len * 4, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+  if (bias && N > 0 && (e = cudaMemcpyAsync(dbias, bias, (size_t)N * 4, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+  st = lba_gemm(dA, dB, dsa, scale_a_len, dsb, scale_b_len, dbias, M, N, K, prod_fmt, acc_fmt, order, chunk, dout, stream);
+  if (st != LBA_OK) return st;
+  if (M * N > 0 && (e = cudaMemcpyAsync(out, dout, (size_t)M * N * 4, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+  return LBA_OK;
+}
+
+size_t lba_conv2d_host_workspace_bytes(int B, int H, int W, int C_in, int C_out, int KH, int KW, int stride_h,
+                                       int stride_w, int pad_h, int pad_w, int scale_x_len, int scale_w_len,
+                                       int has_bias) {
+  ConvGeom g;
+  if (conv_geom(B, H, W, C_in, C_out, KH, KW, stride_h, stride_w, pad_h, pad_w, &g) != LBA_OK) return 0;
+  if (scale_x_len < 0 || scale_w_len < 0) return 0;
+  size_t b = 0;
+  b += round_up((size_t)B * H * W * C_in, 256) + round_up((size_t)C_out * g.K, 256);
+  b += round_up((size_t)scale_x_len * 4, 256) + round_up((size_t)scale_w_len * 4, 256);
+  if (has_bias) b += round_up((size_t)C_out * 4, 256);
+  b += round_up((size_t)g.M * C_out * 4, 256);
+  return b;
+}
+
+int lba_conv2d_host(const uint8_t* x, const uint8_t* w, const float* scale_x, int scale_x_len,
+                    const float* scale_w, int scale_w_len, const float* bias, int B, int H, int W, int C_in,
+                    int C_out, int KH, int KW, int stride_h, int stride_w, int pad_h, int pad_w,
+                    const lba_fmt* prod_fmt, const lba_fmt* acc_fmt, int order, int chunk, float* out,
+                    void* workspace, size_t workspace_bytes, void* stream) {
+  ConvGeom g;
+  int st = conv_geom(B, H, W, C_in, C_out, KH, KW, stride_h, stride_w, pad_h, pad_w, &g);
+  if (st != LBA_OK) return st;
+  if (!x || !w || !out || !scale_x || !scale_w) return LBA_ERR_NULL;
+  if (!(scale_x_len == 1 || scale_x_len == g.M) || !(scale_w_len == 1 || scale_w_len == C_out)) return LBA_ERR_SCALE_LEN;
+  Plan pl;
+  if ((st = make_plan(prod_fmt, acc_fmt, order, chunk, g.K, &pl)) != LBA_OK) return st;
+  const size_t need = lba_conv2d_host_workspace_bytes(B, H, W, C_in, C_out, KH, KW, stride_h, stride_w, pad_h, pad_w,
+                                                      scale_x_len, scale_w_len, bias != nullptr);
+  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255)) return LBA_ERR_WORKSPACE;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t xb = (size_t)B * H * W * C_in, wb = (size_t)C_out * g.K, ob = (size_t)g.M * C_out * 4;
+  uint8_t* ws = (uint8_t*)workspace;
+  uint8_t* dx = ws; ws += round_up(xb, 256);
+  uint8_t* dw = ws; ws += round_up(wb, 256);
+  float* dsx = (float*)ws; ws += round_up((size_t)scale_x_len * 4, 256);
+  float* dsw = (float*)ws; ws += round_up((size_t)scale_w_len * 4, 256);
+  float* dbias = nullptr;
+  if (bias) { dbias = (float*)ws; ws += round_up((size_t)C_out * 4, 256); }
+  float* dout = (float*)ws;
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(dx, x, xb, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(dw, w, wb, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(dsx, scale_x, (size_t)scale_x_len * 4, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(dsw, scale_w, (size_t)scale_w_len * 4, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+  if (bias && (e = cudaMemcpyAsync(dbias, bias, (size_t)C_out * 4, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+  st = lba_conv2d(dx, dw, dsx, scale_x_len, dsw, scale_w_len, dbias, B, H, W, C_in, C_out, KH, KW, stride_h, stride_w,
+                  pad_h, pad_w, prod_fmt, acc_fmt, order, chunk, dout, stream);
+  if (st != LBA_OK) return st;
+  if ((e = cudaMemcpyAsync(out, dout, ob, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+  return LBA_OK;
+}
+
+int lba_count_nan_codes(const uint8_t* codes, int64_t n, unsigned long long* count, void* stream) {
+  if (n < 0) return LBA_ERR_SHAPE;
+  if (!count || (n > 0 && !codes)) return LBA_ERR_NULL;
+  if (n == 0) return LBA_OK;
+  int blocks = (int)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
+  count_nan_codes_kernel<<<blocks, 256, 0, (cudaStream_t)stream>>>(codes, n, count);
+  const cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? LBA_OK : cuda_fail(e);
+}
+
+int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, const lba_fmt* acc_fmt, int order,
+                      int chunk, int is_conv, int vec_ok, char* buf, size_t buf_len) {
+  if (M < 0 || N < 0 || K < 0) return LBA_ERR_SHAPE;
+  Plan pl;
+  const int st = make_plan(prod_fmt, acc_fmt, order, chunk, K, &pl);
+  if (st != LBA_OK) return st;
+  const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, pl.ord);
+  const TileInfo ti = tile_info(tile);
+  const int load = vec_ok ? (is_conv ? LD_CONV_VEC : LD_GEMM_VEC) : LD_ANY;
+  if (buf && buf_len)
+    std::snprintf(buf, buf_len, "tile=%dx%dx%d micro=%dx%d q=%s order=%s load=%s grid=%lldx%lld", ti.bm, ti.bn, BK,
+                  ti.tm, ti.tn, kQmName[pl.qm], kOrdName[pl.ord], kLdName[load], (long long)((M + ti.bm - 1) / ti.bm),
+                  (long long)((N + ti.bn - 1) / ti.bn));
+  return LBA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,3 @@
+#define LBA_QM lba::QM_RNE_WIDE
+#define LBA_ORD lba::ORD_CHUNK_ANY
+#include "lba_family.inc"

@@ -1,0 +1,425 @@
+// LBA contraction kernel for sm_100a: out[m][n] = epilogue(chain_k FMAq(A[m][k], B[n][k], .)).
+//
+// The method rounds after every single addition (Eq. 4 of the paper), so no group of products
+// may be summed exactly first: tensor cores are excluded by definition and the kernel is bound
+// by CUDA-core issue slots.  Everything below exists to keep the per-MAC instruction count low.
+//
+// Carrier arithmetic.  Values are carried in binary32 registers, scaled by a power of two so that
+// the format's underflow threshold R_UF sits at binary32's smallest normal 2^-126:
+//   * product:   p' = x' * w' with x' = x * 2^sx, w' = w * 2^sw, sx + sw = b_prod - 126.  The
+//     product of two E4M3 values has at most 8 significant bits, so it is exact; `mul.ftz` then
+//     flushes exactly the products with |x*w| < R_UF_prod (Eq. 2, second case).
+//   * sum:       t = fma.rz.ftz(p', 2^(b_acc-b_prod), S').  The FMA forms p'*c + S' exactly and
+//     rounds once toward zero to 24 bits; cutting a toward-zero result to M < 24 bits again toward
+//     zero equals cutting the exact sum (truncations compose), so `t & mask` is the floor of Eq. 2
+//     on the exact sum.  `.ftz` flushes exactly the sums below R_UF_acc, because a toward-zero
+//     rounding never moves a value across 2^-126.
+//   * saturation: min.xorsign.abs(t, R_OF') = sign(t) * min(|t|, R_OF'), one instruction.
+// That is 4 instructions per emulated MAC (FMUL, FFMA, LOP3, FMNMX) when Q_prod can neither round
+// nor saturate (M_prod >= 7 and 448^2 < R_OF_prod), which the host proves per call.
+// Nearest-even does not compose with a binary32 rounding, so that mode first builds the
+// round-to-odd value of the exact sum (from the FMA rounded down and up) and rounds that.
+//
+// Data path.  A CTA owns a BM x BN output tile and walks K in slabs of 16 bytes per row: each
+// thread fetches 16-byte row pieces (one 128-bit load), decodes the 16 E4M3 bytes to scaled
+// binary32 once, and stores them k-major into shared memory (double buffered, one barrier per
+// slab).  Each thread keeps a TM x TN register micro-tile of running sums and walks k in order;
+// K is never split across threads, so the paper's accumulation order is kept by construction.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace lba {
+
+enum QMode { QM_FLOOR_FAST = 0, QM_FLOOR_FULL = 1, QM_RNE_FULL = 2, QM_RNE_WIDE = 3, QM_COUNT = 4 };
+enum OrdMode { ORD_SEQ = 0, ORD_CHUNK_SLAB = 1, ORD_CHUNK_ANY = 2, ORD_COUNT = 3 };
+enum LoadMode { LD_GEMM_VEC = 0, LD_CONV_VEC = 1, LD_ANY = 2, LD_COUNT = 3 };
+
+constexpr int BK = 16;  // bytes of K per row per slab = one 128-bit load = one paper-sized chunk
+
+struct QConst {
+  uint32_t mask;     // keeps sign, exponent and the top M mantissa bits
+  uint32_t rne_add;  // nearest-even: 2^(22-M) - 1
+  uint32_t rne_lsb;  // nearest-even: 1, or 0 when M = 23
+  int32_t rne_shift; // nearest-even: 23 - M
+  float sat;         // R_OF in carrier scaling, or FLT_MAX when saturation is unreachable
+};
+
+struct Problem {
+  const uint8_t* A;   // GEMM: [M][K]; conv: x, NHWC
+  const uint8_t* B;   // [N][K]
+  const float* sa;
+  const float* sb;
+  const float* bias;
+  float* out;
+  int64_t M, N, K;
+  int sa_per_row, sb_per_col;
+  int is_conv, H, W, Cin, KH, KW, sh, sw, ph, pw, Hout, Wout;
+  float dec_a, dec_b;  // decode multipliers 2^(120+sx), 2^(120+sw)
+  float c;             // 2^(b_acc' - b_prod'): product carrier -> accumulator carrier
+  float un1, un2;      // un1*un2 = accumulator carrier -> real value
+  QConst qp, qa;
+  int chunk_slabs;     // ORD_CHUNK_SLAB: chunk / BK
+  int chunk;           // ORD_CHUNK_ANY
+};
+
+// ------------------------------------------------------------------ scalar building blocks
+__device__ __forceinline__ float mul_ftz(float a, float b) {
+  float d;
+  asm("mul.rn.ftz.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
+__device__ __forceinline__ float mul_ieee(float a, float b) {  // subnormal operands honoured
+  float d;
+  asm("mul.rn.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
+__device__ __forceinline__ float fma_rz_ftz(float a, float b, float c) {
+  float d;
+  asm("fma.rz.ftz.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float fma_rm(float a, float b, float c) {
+  float d;
+  asm("fma.rm.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float fma_rp(float a, float b, float c) {
+  float d;
+  asm("fma.rp.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float fma_rn(float a, float b, float c) {
+  float d;
+  asm("fma.rn.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// sign(t) * min(|t|, r) for r > 0
+__device__ __forceinline__ float clamp_mag(float t, float r) {
+  float d;
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(d) : "f"(t), "f"(r));
+  return d;
+}
+__device__ __forceinline__ float and_bits(float t, uint32_t m) { return __uint_as_float(__float_as_uint(t) & m); }
+
+// nearest-even cut of a binary32 pattern to M mantissa bits (carry into the exponent is the
+// wanted behaviour); exact when t itself is exact or is the round-to-odd image of the exact value
+__device__ __forceinline__ float rne_bits(float t, const QConst& q) {
+  uint32_t u = __float_as_uint(t);
+  u = u + q.rne_add + ((u >> q.rne_shift) & q.rne_lsb);
+  return __uint_as_float(u & q.mask);
+}
+
+// Q_prod(x*w) in product-carrier scaling.
+template <int QM>
+__device__ __forceinline__ float q_prod(float a, float b, const QConst& qp) {
+  float p = mul_ftz(a, b);  // exact; flushes |x*w| < R_UF_prod
+  if (QM == QM_FLOOR_FULL) {
+    p = clamp_mag(and_bits(p, qp.mask), qp.sat);
+  } else if (QM == QM_RNE_FULL) {
+    p = clamp_mag(rne_bits(p, qp), qp.sat);
+  }
+  return p;
+}
+
+// S <- Q_acc(P*c + S) in accumulator-carrier scaling (c = 1 and P = chunk sum at the second level).
+template <int QM>
+__device__ __forceinline__ float q_acc_fma(float p, float c, float s, const QConst& qa) {
+  if (QM == QM_FLOOR_FAST || QM == QM_FLOOR_FULL) {
+    float t = fma_rz_ftz(p, c, s);
+    return clamp_mag(and_bits(t, qa.mask), qa.sat);
+  } else if (QM == QM_RNE_FULL) {
+    float tz = fma_rz_ftz(p, c, s);   // zero exactly when the exact sum is below R_UF_acc (or is 0)
+    float tm = fma_rm(p, c, s);       // neighbours of the exact sum in binary32
+    float tp = fma_rp(p, c, s);
+    // round-to-odd: if the sum is inexact tm and tp are adjacent and exactly one is odd
+    float ro = (__float_as_uint(tm) & 1u) ? tm : tp;
+    float r = clamp_mag(rne_bits(ro, qa), qa.sat);
+    return tz == 0.0f ? 0.0f : r;
+  } else {  // QM_RNE_WIDE: 24-bit accumulator, nothing of Eq. 2 reachable: one IEEE addition
+    return fma_rn(p, c, s);
+  }
+}
+
+// E4M3 byte (held in the top byte of `top`, lower bytes zero) -> value * mul.
+// (byte & 0x7F) << 20 read as binary32 is value * 2^-120 for normal and subnormal codes alike
+// (E4M3 subnormals land on binary32 subnormals), so one IEEE multiply finishes the decode.
+__device__ __forceinline__ float decode_e4m3_top(uint32_t top, float mul) {
+  float mag = __uint_as_float((top >> 4) & 0x07F00000u);
+  float v = mul_ieee(mag, mul);
+  return __uint_as_float(__float_as_uint(v) | (top & 0x80000000u));
+}
+
+__device__ __forceinline__ uint32_t byte_to_top(uint32_t word, int j) {  // j in 0..3
+  return __byte_perm(word, 0u, (uint32_t)(j << 12) | 0x0444u);
+}
+
+// ------------------------------------------------------------------ the kernel
+template <int BM, int BN, int TM, int TN, int QM, int ORD, int LD>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(const Problem p) {
+  constexpr int NT = (BM / TM) * (BN / TN);
+  constexpr int TX = BN / TN;
+  constexpr int ROWS = BM + BN;
+  constexpr int LPT = (ROWS + NT - 1) / NT;  // 16-byte row pieces fetched per thread per slab
+  constexpr bool CHUNKED = ORD != ORD_SEQ;
+  static_assert(TM == 4 || TM == 8, "micro-tile rows");
+  static_assert(TN == 4 || TN == 8, "micro-tile cols");
+
+  __shared__ __align__(16) float As[2][BK][BM];
+  __shared__ __align__(16) float Bs[2][BK][BN];
+
+  const int tid = threadIdx.x;
+  const int tx = tid % TX, ty = tid / TX;
+  const int64_t m0 = (int64_t)blockIdx.x * BM;
+  const int64_t n0 = (int64_t)blockIdx.y * BN;
+  const int64_t K = p.K;
+  const int nslab = (int)((K + BK - 1) / BK);
+
+  // ---- per-thread loader set-up: which rows of the A and B tiles this thread fetches
+  const uint8_t* row_ptr[LPT];
+  bool row_ok[LPT];
+  int ih0[LPT], iw0[LPT];  // conv: top-left input coordinate of the receptive field
+#pragma unroll
+  for (int l = 0; l < LPT; ++l) {
+    const int r = tid + l * NT;
+    row_ptr[l] = nullptr;
+    row_ok[l] = false;
+    ih0[l] = 0;
+    iw0[l] = 0;
+    if (r < BM) {
+      const int64_t m = m0 + r;
+      if (m < p.M) {
+        row_ok[l] = true;
+        if (LD == LD_GEMM_VEC || (LD == LD_ANY && !p.is_conv)) {
+          row_ptr[l] = p.A + m * K;
+        } else {
+          const int ow = (int)(m % p.Wout);
+          const int64_t t = m / p.Wout;
+          const int oh = (int)(t % p.Hout);
+          const int64_t b = t / p.Hout;
+          ih0[l] = oh * p.sh - p.ph;
+          iw0[l] = ow * p.sw - p.pw;
+          row_ptr[l] = p.A + b * ((int64_t)p.H * p.W * p.Cin);
+        }
+      }
+    } else if (r < ROWS) {
+      const int64_t n = n0 + (r - BM);
+      if (n < p.N) {
+        row_ok[l] = true;
+        row_ptr[l] = p.B + n * K;
+      }
+    }
+  }
+  // conv vector path: position of the current slab inside (kh, kw, c_in)
+  int ld_kh = 0, ld_kw = 0, ld_c0 = 0;
+
+  auto fetch = [&](int slab, uint4 (&raw)[LPT]) {
+    const int64_t k0 = (int64_t)slab * BK;
+#pragma unroll
+    for (int l = 0; l < LPT; ++l) {
+      const int r = tid + l * NT;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (row_ok[l]) {
+        const bool is_a = r < BM;
+        if (LD == LD_GEMM_VEC || (LD == LD_CONV_VEC && !is_a)) {
+          v = __ldg(reinterpret_cast<const uint4*>(row_ptr[l] + k0));
+        } else if (LD == LD_CONV_VEC) {
+          const int ih = ih0[l] + ld_kh, iw = iw0[l] + ld_kw;
+          if (ih >= 0 && ih < p.H && iw >= 0 && iw < p.W)
+            v = __ldg(reinterpret_cast<const uint4*>(row_ptr[l] + ((int64_t)ih * p.W + iw) * p.Cin + ld_c0));
+        } else {  // LD_ANY: byte-wise, any K, any alignment, GEMM or conv
+          uint32_t w4[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+          for (int j = 0; j < BK; ++j) {
+            const int64_t k = k0 + j;
+            uint32_t byte = 0u;
+            if (k < K) {
+              if (!is_a || !p.is_conv) {
+                byte = __ldg(row_ptr[l] + k);
+              } else {
+                const int ci = (int)(k % p.Cin);
+                const int t = (int)(k / p.Cin);
+                const int kw = t % p.KW, kh = t / p.KW;
+                const int ih = ih0[l] + kh, iw = iw0[l] + kw;
+                if (ih >= 0 && ih < p.H && iw >= 0 && iw < p.W)
+                  byte = __ldg(row_ptr[l] + ((int64_t)ih * p.W + iw) * p.Cin + ci);
+              }
+            }
+            w4[j >> 2] |= byte << (8 * (j & 3));
+          }
+          v = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+        }
+      }
+      raw[l] = v;
+    }
+    if (LD == LD_CONV_VEC) {  // advance (kh, kw, c0) to the next slab
+      ld_c0 += BK;
+      if (ld_c0 >= p.Cin) {
+        ld_c0 = 0;
+        if (++ld_kw == p.KW) {
+          ld_kw = 0;
+          ++ld_kh;
+        }
+      }
+    }
+  };
+
+  auto decode_store = [&](const uint4 (&raw)[LPT], int buf) {
+#pragma unroll
+    for (int l = 0; l < LPT; ++l) {
+      const int r = tid + l * NT;
+      if (r < ROWS) {
+        const bool is_a = r < BM;
+        const float mul = is_a ? p.dec_a : p.dec_b;
+        float* dst = is_a ? &As[buf][0][r] : &Bs[buf][0][r - BM];
+        const int stride = is_a ? BM : BN;
+        const uint32_t w4[4] = {raw[l].x, raw[l].y, raw[l].z, raw[l].w};
+#pragma unroll
+        for (int j = 0; j < BK; ++j) dst[j * stride] = decode_e4m3_top(byte_to_top(w4[j >> 2], j & 3), mul);
+      }
+    }
+  };
+
+  // ---- running sums: first hierarchy (or the sequential S) and, in chunked order, the second
+  float acc1[TM][TN];
+  float acc2[CHUNKED ? TM : 1][CHUNKED ? TN : 1];
+#pragma unroll
+  for (int i = 0; i < TM; ++i)
+#pragma unroll
+    for (int j = 0; j < TN; ++j) acc1[i][j] = 0.0f;
+  if (CHUNKED) {
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+      for (int j = 0; j < TN; ++j) acc2[CHUNKED ? i : 0][CHUNKED ? j : 0] = 0.0f;
+  }
+
+  const float cc = p.c;
+  const QConst qp = p.qp, qa = p.qa;
+
+  auto close_chunk = [&]() {  // second hierarchy: T <- Q_acc(C + T), C <- 0
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+      for (int j = 0; j < TN; ++j) {
+        float& t2 = acc2[CHUNKED ? i : 0][CHUNKED ? j : 0];
+        t2 = q_acc_fma<QM>(acc1[i][j], 1.0f, t2, qa);
+        acc1[i][j] = 0.0f;
+      }
+  };
+
+  auto mac_step = [&](int buf, int kk) {
+    float a[TM], b[TN];
+#pragma unroll
+    for (int h = 0; h < TM / 4; ++h) {
+      const float4 v = *reinterpret_cast<const float4*>(&As[buf][kk][h * (BM / 2) + ty * 4]);
+      a[h * 4 + 0] = v.x; a[h * 4 + 1] = v.y; a[h * 4 + 2] = v.z; a[h * 4 + 3] = v.w;
+    }
+#pragma unroll
+    for (int h = 0; h < TN / 4; ++h) {
+      const float4 v = *reinterpret_cast<const float4*>(&Bs[buf][kk][h * (BN / 2) + tx * 4]);
+      b[h * 4 + 0] = v.x; b[h * 4 + 1] = v.y; b[h * 4 + 2] = v.z; b[h * 4 + 3] = v.w;
+    }
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+      for (int j = 0; j < TN; ++j) acc1[i][j] = q_acc_fma<QM>(q_prod<QM>(a[i], b[j], qp), cc, acc1[i][j], qa);
+  };
+
+  // ---- main loop
+  uint4 raw[LPT];
+  int slabs_in_chunk = 0;  // ORD_CHUNK_SLAB
+  int k_in_chunk = 0;      // ORD_CHUNK_ANY
+  if (nslab > 0) {
+    fetch(0, raw);
+    decode_store(raw, 0);
+  }
+  __syncthreads();
+  for (int s = 0; s < nslab; ++s) {
+    const int buf = s & 1;
+    if (s + 1 < nslab) fetch(s + 1, raw);
+    if (ORD == ORD_CHUNK_ANY) {
+      const int kmax = (int)((K - (int64_t)s * BK) < BK ? (K - (int64_t)s * BK) : BK);
+#pragma unroll 1
+      for (int kk = 0; kk < kmax; ++kk) {
+        mac_step(buf, kk);
+        if (++k_in_chunk == p.chunk) {
+          close_chunk();
+          k_in_chunk = 0;
+        }
+      }
+    } else {
+#pragma unroll
+      for (int kk = 0; kk < BK; ++kk) mac_step(buf, kk);
+      if (ORD == ORD_CHUNK_SLAB) {
+        if (++slabs_in_chunk == p.chunk_slabs) {
+          close_chunk();
+          slabs_in_chunk = 0;
+        }
+      }
+    }
+    if (s + 1 < nslab) decode_store(raw, buf ^ 1);
+    __syncthreads();
+  }
+  if (ORD == ORD_CHUNK_SLAB && slabs_in_chunk > 0) close_chunk();
+  if (ORD == ORD_CHUNK_ANY && k_in_chunk > 0) close_chunk();
+
+  // ---- epilogue: back to real values, +0 for every zero, scales and bias in binary32
+  const bool vec_store = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0);
+#pragma unroll
+  for (int i = 0; i < TM; ++i) {
+    const int64_t m = m0 + (i / 4) * (BM / 2) + ty * 4 + (i % 4);
+    if (m >= p.M) continue;
+    const float sa = p.sa[p.sa_per_row ? m : 0];
+#pragma unroll
+    for (int h = 0; h < TN / 4; ++h) {
+      const int64_t n = n0 + h * (BN / 2) + tx * 4;
+      float o[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float s = CHUNKED ? acc2[CHUNKED ? i : 0][CHUNKED ? h * 4 + j : 0] : acc1[i][h * 4 + j];
+        float y = __fmul_rn(__fmul_rn(s, p.un1), p.un2);
+        y = (y == 0.0f) ? 0.0f : y;
+        o[j] = y;
+      }
+      if (n + 3 < p.N && vec_store) {
+        float4 v;
+        float* ov = &v.x;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float sb = p.sb[p.sb_per_col ? n + j : 0];
+          float r = __fmul_rn(__fmul_rn(o[j], sa), sb);
+          if (p.bias) r = __fadd_rn(r, p.bias[n + j]);
+          ov[j] = r;
+        }
+        *reinterpret_cast<float4*>(p.out + m * p.N + n) = v;
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (n + j < p.N) {
+            const float sb = p.sb[p.sb_per_col ? n + j : 0];
+            float r = __fmul_rn(__fmul_rn(o[j], sa), sb);
+            if (p.bias) r = __fadd_rn(r, p.bias[n + j]);
+            p.out[m * p.N + n + j] = r;
+          }
+        }
+      }
+    }
+  }
+}
+
+// Launch entry of one (quantiser mode, order mode) family; defined once per translation unit.
+// tile: 0 = 128x128 (8x8), 1 = 128x64 (8x4), 2 = 64x64 (4x4), 3 = 32x32 (4x4... see table)
+struct TileInfo { int bm, bn, tm, tn; };
+constexpr int TILE_COUNT = 4;
+__host__ inline TileInfo tile_info(int t) {
+  const TileInfo tab[TILE_COUNT] = {{128, 128, 8, 8}, {128, 64, 8, 4}, {64, 64, 4, 4}, {32, 32, 4, 4}};
+  return tab[t];
+}
+
+typedef cudaError_t (*LaunchFn)(int tile, int load, const Problem& p, cudaStream_t stream);
+
+template <int QM, int ORD>
+cudaError_t launch_family(int tile, int load, const Problem& p, cudaStream_t stream);
+
+}  // namespace lba

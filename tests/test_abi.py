@@ -1,0 +1,76 @@
+"""The C ABI without a GPU: the library loads, exports every declared symbol, and rejects bad arguments
+on the host before anything is enqueued."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2401_14110_b200 import binding as lba
+from paper_2401_14110_b200 import LbaFormat, code_domain_formats, ORDER_CHUNKED as CHK, ORDER_SEQUENTIAL as SEQ
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "lba.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(lba_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = lba.load_library()
+    names = _declared_functions()
+    assert "lba_gemm" in names and "lba_conv2d" in names and len(names) >= 10
+    for name in names:
+        assert getattr(lib, name) is not None
+    assert sorted(lba.EXPORTS) == names
+    assert lib.lba_version() == 1
+    assert lib.lba_status_string(0) == b"ok"
+
+
+def test_plan_selection_by_format_and_order():
+    p, a = code_domain_formats(7, 4)
+    assert "q=floor_fast" in lba.describe_plan(64, 64, 576, p, a, SEQ, 16)
+    assert "order=seq" in lba.describe_plan(64, 64, 576, p, a, SEQ, 16)
+    assert "order=chunk_slab" in lba.describe_plan(64, 64, 576, p, a, CHK, 16)
+    assert "order=chunk_slab" in lba.describe_plan(64, 64, 576, p, a, CHK, 32)
+    assert "order=chunk_any" in lba.describe_plan(64, 64, 576, p, a, CHK, 5)
+    assert "order=seq" in lba.describe_plan(64, 64, 576, p, a, CHK, 576)       # one chunk == sequential
+    assert "q=floor_full" in lba.describe_plan(64, 64, 576, LbaFormat(7, 4, 12), LbaFormat(7, 4, 10), CHK, 16)
+    assert "q=floor_full" in lba.describe_plan(64, 64, 576, *code_domain_formats(4, 4), CHK, 16)
+    assert "q=rne_full" in lba.describe_plan(64, 64, 576, *code_domain_formats(7, 4, rounding=1), CHK, 16)
+    assert "q=rne_wide" in lba.describe_plan(64, 64, 576, LbaFormat(23, 8, 127, 1), LbaFormat(23, 8, 127, 1), SEQ, 16)
+    assert "load=conv_vec" in lba.describe_plan(64, 64, 576, p, a, CHK, 16, is_conv=True)
+    assert "load=any" in lba.describe_plan(64, 64, 147, p, a, CHK, 16, is_conv=True, vec_ok=False)
+
+
+@pytest.mark.parametrize("prod,acc,order,chunk,status", [
+    (LbaFormat(0, 4, 8), LbaFormat(7, 4, 8), SEQ, 16, -3),
+    (LbaFormat(7, 9, 8), LbaFormat(7, 4, 8), SEQ, 16, -3),
+    (LbaFormat(7, 4, 500), LbaFormat(7, 4, 8), SEQ, 16, -3),
+    (LbaFormat(7, 4, 8, 3), LbaFormat(7, 4, 8, 3), SEQ, 16, -3),
+    (LbaFormat(7, 4, 8, 0), LbaFormat(7, 4, 8, 1), SEQ, 16, -3),          # mixed rounding rules
+    (LbaFormat(22, 8, 127, 1), LbaFormat(22, 8, 127, 1), SEQ, 16, -3),    # nearest-even with M = 22
+    (LbaFormat(7, 4, 8), LbaFormat(7, 4, 8), 2, 16, -4),
+    (LbaFormat(7, 4, 8), LbaFormat(7, 4, 8), CHK, 0, -4),
+])
+def test_rejected_arguments(prod, acc, order, chunk, status):
+    with pytest.raises(lba.LbaError) as e:
+        lba.describe_plan(8, 8, 8, prod, acc, order, chunk)
+    assert e.value.status == status
+
+
+def test_host_side_checks_run_before_any_cuda_call():
+    lib = lba.load_library()
+    p, a = code_domain_formats(7, 4)
+    pf, af = lba._fmt(p), lba._fmt(a)
+    # null operands, negative sizes, bad scale lengths: all refused without touching a device
+    assert lib.lba_gemm(None, None, None, 1, None, 1, None, 4, 4, 4, C.byref(pf), C.byref(af), 0, 16, None, None) == -1
+    assert lib.lba_gemm(None, None, None, 1, None, 1, None, -1, 4, 4, C.byref(pf), C.byref(af), 0, 16, None, None) == -2
+    fake = C.c_void_p(256)
+    assert lib.lba_gemm(fake, fake, fake, 3, fake, 1, None, 4, 4, 4, C.byref(pf), C.byref(af), 0, 16, fake, None) == -5
+    assert lib.lba_conv2d(fake, fake, fake, 1, fake, 1, None, 1, 2, 2, 3, 4, 5, 5, 1, 1, 0, 0, C.byref(pf),
+                          C.byref(af), 0, 16, fake, None) == -2
+    assert lib.lba_gemm_host_workspace_bytes(4, 4, 16, 1, 1, 0) == 256 * 5
+    assert lib.lba_set_tile_override(9) == -2 and lib.lba_set_tile_override(-1) == 0

@@ -1,0 +1,240 @@
+"""CUDA path versus the CPU oracle, bit for bit, through the C ABI.  Needs a B200."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lba_oracle as orc
+from paper_2401_14110_b200 import binding as lba
+from paper_2401_14110_b200 import synth
+from paper_2401_14110_b200 import (LbaFormat, code_domain_formats, M7E4_PAPER, WIDE, ORDER_SEQUENTIAL as SEQ,
+                                   ORDER_CHUNKED as CHK)
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _bits(a):
+    return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+
+
+def assert_bit_equal(got, want, what=""):
+    got = got.detach().cpu().numpy() if isinstance(got, torch.Tensor) else got
+    g, w = _bits(got).reshape(-1), _bits(want).reshape(-1)
+    bad = np.nonzero(g != w)[0]
+    assert bad.size == 0, (f"{what}: {bad.size} of {g.size} outputs differ; first at {bad[0]}: "
+                           f"gpu={got.reshape(-1)[bad[0]]!r} oracle={np.asarray(want).reshape(-1)[bad[0]]!r}")
+
+
+def gpu_gemm(A, B, sa, sb, bias, prod, acc, order, chunk):
+    d = lambda t: None if t is None else t.to(DEV)
+    return lba.lba_gemm(d(A), d(B), d(sa), d(sb), d(bias), prod, acc, order, chunk)
+
+
+def ref_gemm(A, B, sa, sb, bias, prod, acc, order, chunk):
+    n = lambda t: None if t is None else t.numpy()
+    return orc.gemm(n(A), n(B), n(sa), n(sb), n(bias), prod.as_tuple(), acc.as_tuple(), order, chunk)
+
+
+FORMATS = {
+    "m7e4_code": code_domain_formats(7, 4),                                   # floor_fast
+    "m7e4_paper": M7E4_PAPER,                                                 # Q_prod saturates: floor_full
+    "m4e4": code_domain_formats(4, 4),                                        # Q_prod rounds
+    "m10e5": code_domain_formats(10, 5),
+    "m5e6": code_domain_formats(5, 6),
+    "m4e3_mnist": (LbaFormat(4, 3, 5), LbaFormat(4, 3, 5)),                   # Sec. 4 accumulator
+    "mixed": (LbaFormat(3, 4, 2), LbaFormat(9, 5, 9)),
+    "m7e4_code_rne": code_domain_formats(7, 4, rounding=1),
+    "m4e4_rne": code_domain_formats(4, 4, rounding=1),
+    "m10e6_rne": code_domain_formats(10, 6, rounding=1),
+    "m7e4_paper_rne": (LbaFormat(7, 4, 12, 1), LbaFormat(7, 4, 10, 1)),
+    "mixed_rne": (LbaFormat(7, 4, -2, 1), LbaFormat(5, 4, -4, 1)),            # products off the accumulator grid
+    "m7e4_no_uf": code_domain_formats(7, 4, flags=0),
+    "m4e4_rne_no_uf": code_domain_formats(4, 4, rounding=1, flags=0),
+    "wide_floor": (WIDE, WIDE),
+    "wide_rne": (LbaFormat(23, 8, 127, 1), LbaFormat(23, 8, 127, 1)),
+    "m21_rne": (LbaFormat(21, 8, 127, 1), LbaFormat(21, 8, 127, 1)),
+}
+
+
+def test_config1_single_gemm_all_outputs():
+    # M = N = 64, K = 576, N(0,1) scaled to absmax 448, M7E4, sequential order
+    A, sa, B, sb = synth.gemm_case(64, 64, 576, config=1)
+    prod, acc = code_domain_formats(7, 4)
+    for order in (SEQ, CHK):
+        got = gpu_gemm(A, B, sa, sb, None, prod, acc, order, 16)
+        assert_bit_equal(got, ref_gemm(A, B, sa, sb, None, prod, acc, order, 16), f"config 1 order {order}")
+
+
+@pytest.mark.parametrize("name", list(FORMATS))
+def test_all_e4m3_pairs_k1(name):
+    # every finite pair through one FMAq: out[i][j] = Q_acc(Q_prod(c_i * c_j))
+    prod, acc = FORMATS[name]
+    codes = torch.tensor([c for c in range(256) if (c & 0x7F) != 0x7F], dtype=torch.uint8)[:, None].contiguous()
+    one = torch.ones(1)
+    got = gpu_gemm(codes, codes, one, one, None, prod, acc, SEQ, 16)
+    assert_bit_equal(got, ref_gemm(codes, codes, one, one, None, prod, acc, SEQ, 16), name)
+
+
+@pytest.mark.parametrize("name", list(FORMATS))
+@pytest.mark.parametrize("K", [2, 3, 4, 16, 47, 200])
+def test_random_codes_short_chains(name, K):
+    prod, acc = FORMATS[name]
+    A = synth.random_codes((150, K), 10 + K)
+    B = synth.random_codes((70, K), 20 + K)
+    one = torch.ones(1)
+    for order, chunk in ((SEQ, 16), (CHK, 16), (CHK, 3)):
+        got = gpu_gemm(A, B, one, one, None, prod, acc, order, chunk)
+        assert_bit_equal(got, ref_gemm(A, B, one, one, None, prod, acc, order, chunk), f"{name} K={K} {order}/{chunk}")
+
+
+@pytest.mark.parametrize("tile", [0, 1, 2, 3])
+@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_paper", "m4e4_rne", "wide_rne"])
+def test_every_tile_shape_with_ragged_edges(tile, name):
+    prod, acc = FORMATS[name]
+    lba.set_tile_override(tile)
+    try:
+        for (M, N, K) in ((1, 1, 1), (129, 67, 48), (300, 260, 37), (257, 130, 160)):
+            A, sa, B, sb = synth.gemm_case(M, N, K, config=50 + tile)
+            sa_rows = torch.linspace(0.5, 1.5, M)
+            sb_cols = torch.linspace(0.01, 0.02, N)
+            bias = torch.linspace(-1, 1, N)
+            for order, chunk in ((SEQ, 16), (CHK, 16), (CHK, 32), (CHK, 5)):
+                got = gpu_gemm(A, B, sa_rows, sb_cols, bias, prod, acc, order, chunk)
+                assert_bit_equal(got, ref_gemm(A, B, sa_rows, sb_cols, bias, prod, acc, order, chunk),
+                                 f"tile {tile} {name} {M}x{N}x{K} {order}/{chunk}")
+    finally:
+        lba.set_tile_override(-1)
+
+
+def test_saturation_and_underflow_are_exercised():
+    # make sure the parity cases are not vacuous: both special cases of Eq. 2 occur
+    prod, acc = code_domain_formats(7, 4)
+    A, sa, B, sb = synth.gemm_case(64, 64, 1024, config=7)
+    one = torch.ones(1)
+    a = synth.e4m3_decode(A).numpy().astype(np.float64)
+    b = synth.e4m3_decode(B).numpy().astype(np.float64)
+    prods = np.abs(a[0][None, :] * b)
+    assert ((prods > 0) & (prods < prod.r_uf)).any()          # products that Q_prod flushes
+    # same-sign operands: the running sum climbs to R_OF_acc and stays there
+    Apos, Bpos = A & 0x7F, B & 0x7F
+    for order in (SEQ, CHK):
+        got = gpu_gemm(Apos, Bpos, one, one, None, prod, acc, order, 16).cpu().numpy()
+        assert_bit_equal(got, ref_gemm(Apos, Bpos, one, one, None, prod, acc, order, 16))
+        assert (got == np.float32(acc.r_of)).any()
+    # mixed signs around the top: saturate, come back down, saturate negative
+    Amix = Apos.clone()
+    Amix[:, 512:] |= 0x80
+    got = gpu_gemm(Amix, Bpos, one, one, None, prod, acc, CHK, 16).cpu().numpy()
+    assert_bit_equal(got, ref_gemm(Amix, Bpos, one, one, None, prod, acc, CHK, 16))
+
+
+def test_zero_and_empty_shapes():
+    prod, acc = code_domain_formats(7, 4)
+    one = torch.ones(1)
+    A = synth.random_codes((5, 0), 1)
+    B = synth.random_codes((7, 0), 2)
+    got = gpu_gemm(A, B, one, one, torch.arange(7, dtype=torch.float32), prod, acc, CHK, 16).cpu().numpy()
+    assert got.shape == (5, 7) and np.array_equal(got, np.tile(np.arange(7, dtype=np.float32), (5, 1)))
+    assert gpu_gemm(synth.random_codes((0, 8), 1), synth.random_codes((3, 8), 2), one, one, None, prod, acc, CHK,
+                    16).shape == (0, 3)
+    # negative-zero inputs and exact cancellation give +0
+    A = torch.tensor([[0x80, 0x38, 0xB8, 0x00]], dtype=torch.uint8)       # -0, 1, -1, 0
+    B = torch.tensor([[0x38, 0x40, 0x40, 0x38]], dtype=torch.uint8)       # 1, 2, 2, 1
+    for fmts in ((WIDE, WIDE), FORMATS["wide_rne"], code_domain_formats(7, 4, flags=0)):
+        got = gpu_gemm(A, B, one, one, None, *fmts, SEQ, 16).cpu().numpy()
+        assert got[0, 0] == 0 and not np.signbit(got[0, 0])
+
+
+def test_unaligned_operands_take_the_bytewise_loader():
+    prod, acc = code_domain_formats(7, 4)
+    one = torch.ones(1, device=DEV)
+    Abig = synth.random_codes((40 * 64 + 3,), 3).to(DEV)
+    Bbig = synth.random_codes((33 * 64 + 5,), 4).to(DEV)
+    A = Abig[3:].view(40, 64)          # K % 16 == 0 but the base pointer is odd
+    B = Bbig[5:].view(33, 64)
+    assert A.data_ptr() % 16 != 0
+    got = lba.lba_gemm(A, B, one, one, None, prod, acc, CHK, 16)
+    want = orc.gemm(A.cpu().numpy(), B.cpu().numpy(), 1.0, 1.0, None, prod.as_tuple(), acc.as_tuple(), CHK, 16)
+    assert_bit_equal(got, want)
+
+
+CONV_CASES = [
+    # B, H, W, Cin, Cout, KH, KW, stride, pad
+    (2, 12, 12, 3, 64, 7, 7, (2, 2), (3, 3)),      # stem-like: C_in = 3, K = 147, byte-wise loader
+    (2, 9, 9, 16, 40, 3, 3, (1, 1), (1, 1)),       # vector loader, padding on all sides
+    (1, 14, 14, 64, 130, 3, 3, (2, 2), (1, 1)),    # stride 2
+    (3, 8, 8, 32, 70, 1, 1, (2, 2), (0, 0)),       # 1x1 downsample
+    (1, 7, 9, 5, 3, 3, 2, (2, 1), (0, 2)),         # odd everything
+    (1, 5, 5, 48, 33, 5, 5, (1, 1), (2, 2)),
+]
+
+
+@pytest.mark.parametrize("case", CONV_CASES)
+@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_paper", "m4e4_rne"])
+def test_conv2d_matches_direct_convolution(case, name):
+    B, H, W, Cin, Cout, KH, KW, stride, pad = case
+    prod, acc = FORMATS[name]
+    x = synth.random_codes((B, H, W, Cin), 30)
+    w = synth.random_codes((Cout, KH, KW, Cin), 31)
+    sx = torch.tensor([0.37])
+    sw = torch.linspace(0.5, 2.0, Cout)
+    bias = torch.linspace(-3, 3, Cout)
+    for order, chunk in ((SEQ, 16), (CHK, 16), (CHK, 7)):
+        got = lba.lba_conv2d(x.to(DEV), w.to(DEV), sx.to(DEV), sw.to(DEV), bias.to(DEV), stride, pad, prod, acc,
+                             order, chunk)
+        want = orc.conv2d(x.numpy(), w.numpy(), sx.numpy(), sw.numpy(), bias.numpy(), stride, pad, prod.as_tuple(),
+                          acc.as_tuple(), order, chunk)
+        assert tuple(got.shape) == want.shape
+        assert_bit_equal(got, want, f"{case} {name} {order}/{chunk}")
+
+
+@pytest.mark.parametrize("tile", [0, 1, 2, 3])
+def test_conv2d_every_tile(tile):
+    prod, acc = code_domain_formats(7, 4)
+    lba.set_tile_override(tile)
+    try:
+        for case in CONV_CASES[:3]:
+            B, H, W, Cin, Cout, KH, KW, stride, pad = case
+            x, sx = synth.quantise_per_tensor(synth.gaussian((B, H, W, Cin), 40).relu())
+            w, sw = synth.quantise_per_channel(synth.he_normal((Cout, KH, KW, Cin), KH * KW * Cin, 41))
+            got = lba.lba_conv2d(x.to(DEV), w.to(DEV), sx.to(DEV), sw.to(DEV), None, stride, pad, prod, acc, CHK, 16)
+            want = orc.conv2d(x.numpy(), w.numpy(), sx.numpy(), sw.numpy(), None, stride, pad, prod.as_tuple(),
+                              acc.as_tuple(), CHK, 16)
+            assert_bit_equal(got, want, f"tile {tile} {case}")
+    finally:
+        lba.set_tile_override(-1)
+
+
+def test_host_buffer_entry_points():
+    prod, acc = code_domain_formats(7, 4)
+    A, sa, B, sb = synth.gemm_case(200, 96, 128, config=9)
+    bias = torch.linspace(-1, 1, 96)
+    out = torch.empty((200, 96), dtype=torch.float32).pin_memory()
+    ws = torch.empty(lba.gemm_host_workspace_bytes(200, 96, 128, 1, 1, True), dtype=torch.uint8, device=DEV)
+    lba.lba_gemm_host(A.pin_memory(), B.pin_memory(), sa, sb, bias, prod, acc, CHK, 16, out, ws)
+    torch.cuda.synchronize()
+    assert_bit_equal(out, ref_gemm(A, B, sa, sb, bias, prod, acc, CHK, 16))
+    B_, H, W, Cin, Cout, KH, KW, stride, pad = CONV_CASES[1]
+    x = synth.random_codes((B_, H, W, Cin), 50)
+    w = synth.random_codes((Cout, KH, KW, Cin), 51)
+    one = torch.ones(1)
+    Ho, Wo = lba.conv_out_hw(H, W, KH, KW, stride, pad)
+    out = torch.empty((B_, Ho, Wo, Cout), dtype=torch.float32).pin_memory()
+    ws = torch.empty(lba.conv2d_host_workspace_bytes(B_, H, W, Cin, Cout, KH, KW, stride, pad, 1, 1, False),
+                     dtype=torch.uint8, device=DEV)
+    lba.lba_conv2d_host(x, w, one, one, None, stride, pad, prod, acc, CHK, 16, out, ws)
+    torch.cuda.synchronize()
+    assert_bit_equal(out, orc.conv2d(x.numpy(), w.numpy(), 1.0, 1.0, None, stride, pad, prod.as_tuple(),
+                                     acc.as_tuple(), CHK, 16))
+    with pytest.raises(lba.LbaError) as e:
+        lba.lba_gemm_host(A, B, sa, sb, bias, prod, acc, CHK, 16, torch.empty((200, 96)), ws[:16])
+    assert e.value.status == -7
+
+
+def test_nan_code_counter():
+    codes = synth.random_codes((100000,), 60)
+    assert lba.count_nan_codes(codes.to(DEV)) == 0
+    codes[17] = 0x7F
+    codes[99999] = 0xFF
+    assert lba.count_nan_codes(codes.to(DEV)) == 2
