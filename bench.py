@@ -1,0 +1,372 @@
+#!/usr/bin/env python
+"""Benchmark of the LBA contraction on B200: emulated GMAC/s and fraction of the ALU roofline.
+
+Workload (N = 1 GPU): the ResNet-18 forward convolution stack as implicit LBA GEMMs, batch 32,
+synthetic 224x224x3 N(0,1) images, He-normal weights quantised to E4M3 per output channel, activations
+re-quantised per tensor, M7E4 product and accumulator formats (12-bit accumulator), chunk-16 accumulation
+(the paper's order), floor rounding.  A step is one pass over all 20 convolutions and the final linear
+layer through lba_conv2d / lba_gemm; operands are produced once by a real forward pass (PyTorch glue
+between layers) and stay resident in HBM.  With N > 1 every rank runs the same step on its own batch
+(rows of the implicit GEMM are independent; no collective on the data path): weak scaling.
+
+One JSON line is printed by rank 0.  `--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "emulated_lba_gmacs"
+UNIT = "GMAC/s"
+WORKLOAD = "resnet18_fwd_conv_stack_b32_224_m7e4_chunk16"
+BATCH = 32
+CONFIG_ID = 2
+
+# ALU roofline constants for sm_100: per SM and clock, 128 lanes can be issued and the integer/logic/min-max
+# pipe executes 64 lanes; the fast floor path needs 2 instructions of that pipe per emulated MAC
+# (mantissa mask and magnitude clamp).
+ISSUE_LANES_PER_SM_CLK = 128
+ALU_PIPE_LANES_PER_SM_CLK = 64
+ALU_PIPE_INSTR_PER_MAC = 2.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-baseline-macs", type=float, default=1.5e9,
+                    help="size of the oracle sample timed for cpu_baseline (emulated MACs)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, index):
+        self.index = index
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+
+    def _run(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={q}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                f = [x.strip() for x in out.strip().split(",")]
+                self.samples.append(float(f[0]))
+                self.max_mhz = float(f[1])
+                for n, v in zip(names, f[2:]):
+                    if v.lower().startswith("active"):
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            self._stop.wait(0.05)
+
+    def start(self):
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join(timeout=10)
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def formats():
+    from paper_2401_14110_b200 import code_domain_formats
+    return code_domain_formats(7, 4)
+
+
+def build_calls(device):
+    from paper_2401_14110_b200 import binding as lba, workloads, ORDER_CHUNKED
+    prod, acc = formats()
+
+    def conv_fn(x, w, sx, sw, stride, pad):
+        return lba.lba_conv2d(x, w, sx, sw, None, stride, pad, prod, acc, ORDER_CHUNKED, 16)
+
+    def gemm_fn(a, b, sa, sb):
+        return lba.lba_gemm(a, b, sa, sb, None, prod, acc, ORDER_CHUNKED, 16)
+
+    calls, _ = workloads.build_resnet_calls("resnet18", BATCH, CONFIG_ID, device, conv_fn, gemm_fn)
+    for c in calls:
+        m, n, _ = c.gemm_shape
+        c.out = torch.empty((m, n), dtype=torch.float32, device=device)
+    return calls
+
+
+def run_step(calls, events=None):
+    from paper_2401_14110_b200 import binding as lba, ORDER_CHUNKED
+    prod, acc = formats()
+    for i, c in enumerate(calls):
+        if events is not None:
+            events[i][0].record()
+        if c.kind == "conv":
+            lba.lba_conv2d(c.x, c.w, c.sx, c.sw, None, c.stride, c.pad, prod, acc, ORDER_CHUNKED, 16, out=c.out_nhwc)
+        else:
+            lba.lba_gemm(c.x, c.w, c.sx, c.sw, None, prod, acc, ORDER_CHUNKED, 16, out=c.out)
+        if events is not None:
+            events[i][1].record()
+
+
+def describe(c):
+    from paper_2401_14110_b200 import binding as lba, ORDER_CHUNKED
+    prod, acc = formats()
+    m, n, k = c.gemm_shape
+    vec = (c.x.shape[-1] % 16 == 0) if c.kind == "conv" else (k % 16 == 0)
+    return lba.describe_plan(m, n, k, prod, acc, ORDER_CHUNKED, 16, is_conv=c.kind == "conv", vec_ok=vec)
+
+
+def cpu_baseline(calls, target_macs):
+    """Time the oracle, as it stands, on a bounded sample: seeded 16x16 output tiles of several layers."""
+    from oracle import lba_oracle as orc
+    from paper_2401_14110_b200 import synth, ORDER_CHUNKED
+    prod, acc = formats()
+    picks = [c for c in calls if c.kind == "conv"][1::4] + [calls[0]]
+    per_layer = target_macs / len(picks)
+    jobs = []
+    for i, c in enumerate(picks):
+        m, n, k = c.gemm_shape
+        tiles = max(1, int(per_layer / (256 * k)))
+        ms, ns = synth.sample_tiles(m, n, tiles, 16, 777 + i)
+        jobs.append((c, c.x.cpu().numpy(), c.w.cpu().numpy(), c.sx.cpu().numpy(), c.sw.cpu().numpy(), ms, ns, k))
+    cores = orc.default_threads()
+    orc.lib()
+    t0 = time.perf_counter()
+    macs = 0
+    for c, x, w, sx, sw, ms, ns, k in jobs:
+        orc.conv2d_points(x, w, sx, sw, None, c.stride, c.pad, prod.as_tuple(), acc.as_tuple(), ORDER_CHUNKED, 16,
+                          ms, ns, nthreads=cores)
+        macs += len(ms) * k
+    dt = time.perf_counter() - t0
+    return {"value": macs / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{len(jobs)} layers x seeded 16x16 output tiles, {macs:.3g} MACs in {dt:.1f} s",
+            "macs": macs, "seconds": dt}
+
+
+def reference_arm(args):
+    """The oracle timed on the host cores; each step is a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import lba_oracle as orc
+    from paper_2401_14110_b200 import synth, workloads, ORDER_CHUNKED
+    prod, acc = formats()
+    specs = workloads.resnet18_convs()
+    picks = [specs[1], specs[6], specs[11], specs[16]]       # one 3x3 convolution from each stage
+    cores = orc.default_threads()
+    jobs = []
+    for i, s in enumerate(picks):
+        hw = s.h_in
+        x, sx = synth.quantise_per_tensor(synth.gaussian((2, hw, hw, s.c_in), synth.seed_for(CONFIG_ID, 500 + i)).relu())
+        w, sw = synth.quantise_per_channel(synth.he_normal((s.c_out, s.k, s.k, s.c_in), s.k * s.k * s.c_in,
+                                                           synth.seed_for(CONFIG_ID, 600 + i)))
+        m, n, k = 2 * s.h_out * s.h_out, s.c_out, s.k * s.k * s.c_in
+        tiles = max(1, int(5e7 / (256 * k)))
+        ms, ns = synth.sample_tiles(m, n, tiles, 16, 900 + i)
+        jobs.append((s, x.numpy(), w.numpy(), sx.numpy(), sw.numpy(), ms, ns, k))
+    step_macs = sum(len(j[5]) * j[7] for j in jobs)
+
+    def step():
+        for s, x, w, sx, sw, ms, ns, k in jobs:
+            orc.conv2d_points(x, w, sx, sw, None, (s.stride, s.stride), (s.pad, s.pad), prod.as_tuple(),
+                              acc.as_tuple(), ORDER_CHUNKED, 16, ms, ns, nthreads=cores)
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = step_macs * args.steps / dt / 1e9
+    sample = f"per step: seeded 16x16 output tiles of 4 ResNet-18 3x3 convolutions, {step_macs:.3g} MACs"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int128 exact dyadic (CPU)", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        reference_arm(args)
+        return
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the LBA library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    from paper_2401_14110_b200 import binding as lba, ORDER_CHUNKED
+    lba.load_library()
+    prod, acc = formats()
+    calls = build_calls(device)
+    for c in calls:
+        if c.kind == "conv":
+            b, h, w, _ = c.x.shape
+            ho, wo = lba.conv_out_hw(h, w, c.w.shape[1], c.w.shape[2], c.stride, c.pad)
+            c.out_nhwc = c.out.view(b, ho, wo, c.w.shape[0])
+    step_macs = sum(c.macs for c in calls)
+    launches_per_step = len(calls)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        run_step(calls)
+    barrier()
+
+    # ---- timed region: K steps, per-launch CUDA events on the launching stream
+    events = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in calls]
+              for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record()
+    for s in range(args.steps):
+        run_step(calls, events[s])
+    stop.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = start.elapsed_time(stop)
+    if dist is not None:
+        t = torch.tensor([total_ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * step_macs / (ms_per_step * 1e-3) / 1e9
+
+    # ---- per-kernel accounting from the per-launch events
+    per_call_ms = [statistics.mean(events[s][i][0].elapsed_time(events[s][i][1]) for s in range(args.steps))
+                   for i in range(len(calls))]
+    by_kernel = {}
+    for c, ms in zip(calls, per_call_ms):
+        d = describe(c)
+        key = " ".join(p for p in d.split() if not p.startswith("grid="))
+        e = by_kernel.setdefault(key, {"ms": 0.0, "macs": 0, "launches": 0})
+        e["ms"] += ms
+        e["macs"] += c.macs
+        e["launches"] += 1
+    dom_key, dom = max(by_kernel.items(), key=lambda kv: kv[1]["ms"])
+    sm_count = torch.cuda.get_device_properties(device).multi_processor_count
+    mhz = clocks["sm_mhz"] or clocks["sm_max_mhz"] or 1965.0
+    alu_pipe_bound = sm_count * ALU_PIPE_LANES_PER_SM_CLK * mhz * 1e6 / ALU_PIPE_INSTR_PER_MAC / 1e9
+    achieved = dom["macs"] / (dom["ms"] * 1e-3) / 1e9
+    roofline = {
+        "bound": "alu", "achieved": achieved, "peak": alu_pipe_bound, "unit": UNIT, "frac": achieved / alu_pipe_bound,
+        "traffic": None,
+        "kernel": dom_key, "kernel_launches_per_step": dom["launches"], "kernel_ms_per_step": dom["ms"],
+        "kernel_share_of_step": dom["ms"] / sum(per_call_ms),
+        "peak_derivation": f"{sm_count} SMs x {ALU_PIPE_LANES_PER_SM_CLK} integer/logic lanes per clock x {mhz:.0f} MHz "
+                           f"(median sampled) / {ALU_PIPE_INSTR_PER_MAC:g} such instructions per emulated MAC",
+        "whole_step_frac_of_peak": (step_macs / (sum(per_call_ms) * 1e-3) / 1e9) / alu_pipe_bound,
+    }
+
+    # ---- end to end through the host-buffer C entry points
+    e2e = None
+    if not args.no_e2e:
+        host = []
+        ws_bytes = 0
+        h2d = d2h = 0
+        for c in calls:
+            hx, hw_, hsx, hsw = (t.cpu().pin_memory() for t in (c.x, c.w, c.sx, c.sw))
+            hout = torch.empty(c.out.shape if c.kind == "gemm" else c.out_nhwc.shape, dtype=torch.float32).pin_memory()
+            if c.kind == "conv":
+                b, h, w, cin = c.x.shape
+                cout, kh, kw, _ = c.w.shape
+                need = lba.conv2d_host_workspace_bytes(b, h, w, cin, cout, kh, kw, c.stride, c.pad, 1, cout, False)
+            else:
+                m, n, k = c.gemm_shape
+                need = lba.gemm_host_workspace_bytes(m, n, k, 1, n, False)
+            ws_bytes = max(ws_bytes, need)
+            h2d += hx.numel() + hw_.numel() + 4 * (hsx.numel() + hsw.numel())
+            d2h += 4 * hout.numel()
+            host.append((c, hx, hw_, hsx, hsw, hout))
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
+
+        def e2e_step():
+            for c, hx, hw_, hsx, hsw, hout in host:
+                if c.kind == "conv":
+                    lba.lba_conv2d_host(hx, hw_, hsx, hsw, None, c.stride, c.pad, prod, acc, ORDER_CHUNKED, 16, hout, ws)
+                else:
+                    lba.lba_gemm_host(hx, hw_, hsx, hsw, None, prod, acc, ORDER_CHUNKED, 16, hout, ws)
+        e2e_steps = max(2, min(args.steps, 5))
+        e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e_step()
+        barrier()
+        e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
+        if dist is not None:
+            t = torch.tensor([e2e_ms], device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e = {"value": world * step_macs / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
+               "api": "lba_conv2d_host / lba_gemm_host (pinned host buffers, caller-owned device workspace)"}
+        del ws, host
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(calls, args.cpu_baseline_macs)
+
+    if rank == 0:
+        working_set = sum(c.x.numel() + c.w.numel() + 4 * c.out.numel() for c in calls)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "fp8_e4m3 in, 12-bit M7E4 accumulator emulated in f32 registers, f32 out",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "batch_per_gpu": BATCH, "lba_calls_per_step": launches_per_step,
+                       "macs_per_step_per_gpu": step_macs, "prod_fmt": list(prod.as_tuple()),
+                       "acc_fmt": list(acc.as_tuple()), "order": "chunked", "chunk": 16,
+                       "l2": f"no flush: each step streams {working_set / 1e6:.0f} MB of distinct operands and "
+                             f"outputs, larger than the 126 MB L2",
+                       "parallelism": f"dp{world} (batch sharded, weights replicated, no collective)"},
+            "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
+            "kernels": {k: {"ms_per_step": v["ms"], "launches_per_step": v["launches"],
+                            "gmacs": v["macs"] / (v["ms"] * 1e-3) / 1e9} for k, v in by_kernel.items()},
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
