@@ -50,6 +50,7 @@ constexpr int kMinProductExp = -18;            // every product, hence every sum
 struct Plan {
   int qm, ord;
   float dec_a, dec_b, c, un1, un2;
+  float pk_a, pk_b, nrm_scale, inv_top;
   QConst qp, qa;
   int chunk_slabs, chunk;
 };
@@ -141,6 +142,25 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
   const int u1 = (-ka) / 2, u2 = (-ka) - u1;
   pl->un1 = (float)std::ldexp(1.0, u1);
   pl->un2 = (float)std::ldexp(1.0, u2);
+  // packed floor kernel: operands decoded by the hardware converter, then scaled by 2^sx, 2^sw; row
+  // norms and |S| are measured as fractions of 2^(e_max_acc + 1), the first magnitude the mantissa
+  // mask alone would not bring back to R_OF.  A scale that binary32 cannot hold switches the
+  // clamp-free path off (infinite norms) rather than risk an underestimate.
+  pl->pk_a = (float)std::ldexp(1.0, sx);
+  pl->pk_b = (float)std::ldexp(1.0, sw);
+  if (!a_sat) {
+    pl->nrm_scale = 0.0f;
+    pl->inv_top = 0.0f;
+  } else {
+    const int e1 = -(a_emax + 1), e2 = -ka - (a_emax + 1);
+    if (e1 < -140 || e1 > 127 || e2 < -126 || e2 > 127) {
+      pl->nrm_scale = INFINITY;
+      pl->inv_top = 0.0f;
+    } else {
+      pl->nrm_scale = (float)std::ldexp(1.0, e1);
+      pl->inv_top = (float)std::ldexp(1.0, e2);
+    }
+  }
 
   // ---- order mode
   pl->chunk = chunk;
@@ -207,6 +227,10 @@ void apply_plan(Problem* p, const Plan& pl) {
   p->qa = pl.qa;
   p->chunk_slabs = pl.chunk_slabs;
   p->chunk = pl.chunk;
+  p->pk_a = pl.pk_a;
+  p->pk_b = pl.pk_b;
+  p->nrm_scale = pl.nrm_scale;
+  p->inv_top = pl.inv_top;
 }
 
 bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0; }

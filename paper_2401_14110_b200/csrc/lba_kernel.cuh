@@ -27,6 +27,7 @@
 // K is never split across threads, so the paper's accumulation order is kept by construction.
 #pragma once
 #include <cstdint>
+#include <type_traits>
 #include <cuda_runtime.h>
 
 namespace lba {
@@ -61,6 +62,10 @@ struct Problem {
   QConst qp, qa;
   int chunk_slabs;     // ORD_CHUNK_SLAB: chunk / BK
   int chunk;           // ORD_CHUNK_ANY
+  // packed floor kernel only
+  float pk_a, pk_b;    // 2^sx, 2^sw: decoded value -> product-carrier operand
+  float nrm_scale;     // 2^-(e_max_acc + 1), or 0 when the accumulator cannot saturate
+  float inv_top;       // accumulator carrier -> fraction of 2^(e_max_acc + 1)
 };
 
 // ------------------------------------------------------------------ scalar building blocks
@@ -154,66 +159,56 @@ __device__ __forceinline__ uint32_t byte_to_top(uint32_t word, int j) {  // j in
   return __byte_perm(word, 0u, (uint32_t)(j << 12) | 0x0444u);
 }
 
-// ------------------------------------------------------------------ the kernel
-template <int BM, int BN, int TM, int TN, int QM, int ORD, int LD>
-__global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(const Problem p) {
-  constexpr int NT = (BM / TM) * (BN / TN);
-  constexpr int TX = BN / TN;
-  constexpr int ROWS = BM + BN;
-  constexpr int LPT = (ROWS + NT - 1) / NT;  // 16-byte row pieces fetched per thread per slab
-  constexpr bool CHUNKED = ORD != ORD_SEQ;
-  static_assert(TM == 4 || TM == 8, "micro-tile rows");
-  static_assert(TN == 4 || TN == 8, "micro-tile cols");
-
-  __shared__ __align__(16) float As[2][BK][BM];
-  __shared__ __align__(16) float Bs[2][BK][BN];
-
-  const int tid = threadIdx.x;
-  const int tx = tid % TX, ty = tid / TX;
-  const int64_t m0 = (int64_t)blockIdx.x * BM;
-  const int64_t n0 = (int64_t)blockIdx.y * BN;
-  const int64_t K = p.K;
-  const int nslab = (int)((K + BK - 1) / BK);
-
-  // ---- per-thread loader set-up: which rows of the A and B tiles this thread fetches
+// ------------------------------------------------------------------ operand fetch
+// Each thread fetches, per slab, 16-byte pieces of the rows r = tid + l*NT of the CTA's A tile
+// (r < BM) and B tile (BM <= r < BM + BN).  Rows past the matrix edge and padded convolution taps
+// read as zero bytes, i.e. the value 0.
+template <int BM, int BN, int NT, int LD>
+struct RowLoader {
+  static constexpr int ROWS = BM + BN;
+  static constexpr int LPT = (ROWS + NT - 1) / NT;
   const uint8_t* row_ptr[LPT];
   bool row_ok[LPT];
-  int ih0[LPT], iw0[LPT];  // conv: top-left input coordinate of the receptive field
+  int ih0[LPT], iw0[LPT];               // conv: top-left input coordinate of the receptive field
+  int ld_kh = 0, ld_kw = 0, ld_c0 = 0;  // conv vector path: position of the next slab inside (kh, kw, c_in)
+
+  __device__ __forceinline__ void init(const Problem& p, int tid, int64_t m0, int64_t n0) {
 #pragma unroll
-  for (int l = 0; l < LPT; ++l) {
-    const int r = tid + l * NT;
-    row_ptr[l] = nullptr;
-    row_ok[l] = false;
-    ih0[l] = 0;
-    iw0[l] = 0;
-    if (r < BM) {
-      const int64_t m = m0 + r;
-      if (m < p.M) {
-        row_ok[l] = true;
-        if (LD == LD_GEMM_VEC || (LD == LD_ANY && !p.is_conv)) {
-          row_ptr[l] = p.A + m * K;
-        } else {
-          const int ow = (int)(m % p.Wout);
-          const int64_t t = m / p.Wout;
-          const int oh = (int)(t % p.Hout);
-          const int64_t b = t / p.Hout;
-          ih0[l] = oh * p.sh - p.ph;
-          iw0[l] = ow * p.sw - p.pw;
-          row_ptr[l] = p.A + b * ((int64_t)p.H * p.W * p.Cin);
+    for (int l = 0; l < LPT; ++l) {
+      const int r = tid + l * NT;
+      row_ptr[l] = nullptr;
+      row_ok[l] = false;
+      ih0[l] = 0;
+      iw0[l] = 0;
+      if (r < BM) {
+        const int64_t m = m0 + r;
+        if (m < p.M) {
+          row_ok[l] = true;
+          if (LD == LD_GEMM_VEC || (LD == LD_ANY && !p.is_conv)) {
+            row_ptr[l] = p.A + m * p.K;
+          } else {
+            const int ow = (int)(m % p.Wout);
+            const int64_t t = m / p.Wout;
+            const int oh = (int)(t % p.Hout);
+            const int64_t b = t / p.Hout;
+            ih0[l] = oh * p.sh - p.ph;
+            iw0[l] = ow * p.sw - p.pw;
+            row_ptr[l] = p.A + b * ((int64_t)p.H * p.W * p.Cin);
+          }
         }
-      }
-    } else if (r < ROWS) {
-      const int64_t n = n0 + (r - BM);
-      if (n < p.N) {
-        row_ok[l] = true;
-        row_ptr[l] = p.B + n * K;
+      } else if (r < ROWS) {
+        const int64_t n = n0 + (r - BM);
+        if (n < p.N) {
+          row_ok[l] = true;
+          row_ptr[l] = p.B + n * p.K;
+        }
       }
     }
   }
-  // conv vector path: position of the current slab inside (kh, kw, c_in)
-  int ld_kh = 0, ld_kw = 0, ld_c0 = 0;
 
-  auto fetch = [&](int slab, uint4 (&raw)[LPT]) {
+  // slabs must be requested in increasing order, each once (the conv vector path keeps a cursor)
+  __device__ __forceinline__ void fetch(const Problem& p, int tid, int slab, uint4 (&raw)[LPT]) {
+    const int64_t K = p.K;
     const int64_t k0 = (int64_t)slab * BK;
 #pragma unroll
     for (int l = 0; l < LPT; ++l) {
@@ -262,7 +257,33 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
         }
       }
     }
-  };
+  }
+};
+
+// ------------------------------------------------------------------ the kernel
+template <int BM, int BN, int TM, int TN, int QM, int ORD, int LD>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(const Problem p) {
+  constexpr int NT = (BM / TM) * (BN / TN);
+  constexpr int TX = BN / TN;
+  constexpr int ROWS = BM + BN;
+  constexpr int LPT = (ROWS + NT - 1) / NT;  // 16-byte row pieces fetched per thread per slab
+  constexpr bool CHUNKED = ORD != ORD_SEQ;
+  static_assert(TM == 4 || TM == 8, "micro-tile rows");
+  static_assert(TN == 4 || TN == 8, "micro-tile cols");
+
+  __shared__ __align__(16) float As[2][BK][BM];
+  __shared__ __align__(16) float Bs[2][BK][BN];
+
+  const int tid = threadIdx.x;
+  const int tx = tid % TX, ty = tid / TX;
+  const int64_t m0 = (int64_t)blockIdx.x * BM;
+  const int64_t n0 = (int64_t)blockIdx.y * BN;
+  const int64_t K = p.K;
+  const int nslab = (int)((K + BK - 1) / BK);
+
+  RowLoader<BM, BN, NT, LD> loader;
+  loader.init(p, tid, m0, n0);
+  auto fetch = [&](int slab, uint4 (&raw)[LPT]) { loader.fetch(p, tid, slab, raw); };
 
   auto decode_store = [&](const uint4 (&raw)[LPT], int buf) {
 #pragma unroll
@@ -406,6 +427,285 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
       }
     }
   }
+}
+
+// ------------------------------------------------------------------ packed floor kernel
+// The fast floor quantiser (Q_prod reduced to its flush, floor rounding) on the packed binary32
+// instructions of sm_100: two neighbouring outputs of a row share one 64-bit register pair, so
+// the product and the sum of two emulated MACs cost one `mul.ftz.f32x2` and one `fma.rz.ftz.f32x2`,
+// followed by one mantissa mask per output.  The magnitude clamp of Eq. 2 is left out of a slab
+// whenever it provably cannot act there:
+//   |S_i| <= |S_start| + sum_k |x_k w_k| <= |S_start| + ||x||_2 ||w||_2        (floor never grows |.|)
+// so if that bound stays below 2^(e_max+1) every masked sum is already <= R_OF.  The loader
+// computes the squared 2-norm of every 16-byte row piece while decoding it; the largest A-row and
+// B-row norms of the slab give one bound per CTA, and each thread carries an upper bound `u` of
+// its own |S| (as a fraction of 2^(e_max+1)), refreshed from the registers when it gets too loose.
+// A warp whose bound fails runs the same slab with the clamp.  Results are identical either way.
+typedef unsigned long long u64;
+constexpr int KUNROLL = 16;  // k-steps unrolled in the packed slab body (the whole slab: measured fastest)
+
+__device__ __forceinline__ u64 pack2(float lo, float hi) {
+  u64 d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 mul2_ftz(u64 a, u64 b) {
+  u64 d;
+  asm("mul.rn.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ u64 fma2_rz_ftz(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rz.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 add2_rz_ftz(u64 a, u64 b) {
+  u64 d;
+  asm("add.rz.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// two E4M3 bytes (low 16 bits of `pair`) -> their exact values, by the hardware converter
+__device__ __forceinline__ void e4m3x2_to_f32(uint32_t pair, float& v0, float& v1) {
+  asm("{\n\t.reg .b16 c, lo, hi;\n\t.reg .b32 h;\n\t"
+      "cvt.u16.u32 c, %2;\n\t"
+      "cvt.rn.f16x2.e4m3x2 h, c;\n\t"
+      "mov.b32 {lo, hi}, h;\n\t"
+      "cvt.f32.f16 %0, lo;\n\t"
+      "cvt.f32.f16 %1, hi;\n\t}"
+      : "=f"(v0), "=f"(v1)
+      : "r"(pair));
+}
+
+template <int BM, int BN, int TM, int TN, int ORD, int LD>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_kernel(const Problem p) {
+  constexpr int NT = (BM / TM) * (BN / TN);
+  constexpr int TX = BN / TN;
+  constexpr int ROWS = BM + BN;
+  constexpr int LPT = (ROWS + NT - 1) / NT;
+  constexpr int PN = TN / 2;  // register pairs per micro-tile row
+  constexpr bool CHUNKED = ORD == ORD_CHUNK_SLAB;
+  static_assert(ORD == ORD_SEQ || ORD == ORD_CHUNK_SLAB, "order");
+  static_assert(TM == 4 || TM == 8, "micro-tile rows");
+  static_assert(TN == 4 || TN == 8, "micro-tile cols");
+  static_assert(BM % 32 == 0 && BN % 32 == 0, "a warp loads rows of one operand only");
+
+  // A is stored twice, {a, a}, so that a 64-bit shared load yields the packed multiplier directly
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  typedef float2 (*AsT)[BK][BM];
+  typedef float (*BsT)[BK][BN];
+  AsT As = reinterpret_cast<AsT>(smem_raw);
+  BsT Bs = reinterpret_cast<BsT>(smem_raw + sizeof(float2) * 2 * BK * BM);
+  // largest normalised squared row norm of the slab, as binary32 bits (non-negative, so they order
+  // like integers): [slab % 3][0 = A, 1 = B]; three cells so that one can be cleared while the
+  // neighbours are read and filled
+  unsigned (*nrm)[2] = reinterpret_cast<unsigned (*)[2]>(smem_raw + sizeof(float2) * 2 * BK * BM + sizeof(float) * 2 * BK * BN);
+
+  const int tid = threadIdx.x;
+  const int tx = tid % TX, ty = tid / TX;
+  const int64_t m0 = (int64_t)blockIdx.x * BM;
+  const int64_t n0 = (int64_t)blockIdx.y * BN;
+  const int nslab = (int)((p.K + BK - 1) / BK);
+
+  RowLoader<BM, BN, NT, LD> loader;
+  loader.init(p, tid, m0, n0);
+
+  auto decode_store = [&](const uint4 (&raw)[LPT], int buf, int cell) {
+#pragma unroll
+    for (int l = 0; l < LPT; ++l) {
+      const int r = tid + l * NT;
+      if (r < ROWS) {  // uniform per warp: BM, BN and NT are multiples of 32
+        const bool is_a = r < BM;
+        const float mul = is_a ? p.pk_a : p.pk_b;
+        const uint32_t w4[4] = {raw[l].x, raw[l].y, raw[l].z, raw[l].w};
+        float n2 = 0.0f;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          float v[4];
+          e4m3x2_to_f32(w4[q], v[0], v[1]);
+          e4m3x2_to_f32(w4[q] >> 16, v[2], v[3]);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            n2 = fma_rn(v[j], v[j], n2);
+            const float s = mul_ieee(v[j], mul);
+            if (is_a) As[buf][q * 4 + j][r] = make_float2(s, s);
+            else Bs[buf][q * 4 + j][r - BM] = s;
+          }
+        }
+        const unsigned m = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(n2 * p.nrm_scale));
+        if ((tid & 31) == 0) atomicMax(&nrm[cell][is_a ? 0 : 1], m);
+      }
+    }
+  };
+
+  u64 acc1[TM][PN];
+  u64 acc2[CHUNKED ? TM : 1][CHUNKED ? PN : 1];
+#pragma unroll
+  for (int i = 0; i < TM; ++i)
+#pragma unroll
+    for (int j = 0; j < PN; ++j) acc1[i][j] = 0ull;
+  if (CHUNKED) {
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+      for (int j = 0; j < PN; ++j) acc2[CHUNKED ? i : 0][CHUNKED ? j : 0] = 0ull;
+  }
+
+  const u64 cc2 = pack2(p.c, p.c);
+  const uint32_t mask = p.qa.mask;
+  const float sat = p.qa.sat;
+
+  // one slab of 16 k-steps; CLAMP selects whether the magnitude clamp of Eq. 2 is applied
+  auto slab_body = [&](int buf, auto clamp_tag) {
+    constexpr bool CLAMP = decltype(clamp_tag)::value;
+#pragma unroll KUNROLL
+    for (int kk = 0; kk < BK; ++kk) {
+      u64 a2[TM], b2[PN];
+#pragma unroll
+      for (int h = 0; h < TM / 4; ++h) {
+        const ulonglong2* src = reinterpret_cast<const ulonglong2*>(&As[buf][kk][h * (BM / 2) + ty * 4]);
+        const ulonglong2 v0 = src[0], v1 = src[1];
+        a2[h * 4 + 0] = v0.x; a2[h * 4 + 1] = v0.y; a2[h * 4 + 2] = v1.x; a2[h * 4 + 3] = v1.y;
+      }
+#pragma unroll
+      for (int h = 0; h < TN / 4; ++h) {
+        const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(&Bs[buf][kk][h * (BN / 2) + tx * 4]);
+        b2[h * 2 + 0] = v.x; b2[h * 2 + 1] = v.y;
+      }
+#pragma unroll
+      for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < PN; ++j) {
+          const u64 t = fma2_rz_ftz(mul2_ftz(a2[i], b2[j]), cc2, acc1[i][j]);
+          float lo, hi;
+          unpack2(t, lo, hi);
+          lo = and_bits(lo, mask);
+          hi = and_bits(hi, mask);
+          if (CLAMP) {
+            lo = clamp_mag(lo, sat);
+            hi = clamp_mag(hi, sat);
+          }
+          acc1[i][j] = pack2(lo, hi);
+        }
+    }
+  };
+
+  auto close_chunk = [&]() {  // second hierarchy: T <- Q_acc(C + T), C <- 0 (always clamped: once per chunk)
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+      for (int j = 0; j < PN; ++j) {
+        u64& t2 = acc2[CHUNKED ? i : 0][CHUNKED ? j : 0];
+        float lo, hi;
+        unpack2(add2_rz_ftz(acc1[i][j], t2), lo, hi);
+        t2 = pack2(clamp_mag(and_bits(lo, mask), sat), clamp_mag(and_bits(hi, mask), sat));
+        acc1[i][j] = 0ull;
+      }
+  };
+
+  if (tid < 6) nrm[tid >> 1][tid & 1] = 0u;
+  __syncthreads();
+  uint4 raw[LPT];
+  if (nslab > 0) {
+    loader.fetch(p, tid, 0, raw);
+    decode_store(raw, 0, 0);
+  }
+  __syncthreads();
+
+  float u = 0.0f;  // upper bound of max |acc1| of this thread, as a fraction of 2^(e_max + 1)
+  int slabs_in_chunk = 0;
+  int cell = 0;    // s % 3
+  for (int s = 0; s < nslab; ++s) {
+    const int buf = s & 1;
+    const int cell_next = cell == 2 ? 0 : cell + 1;
+    const int cell_clear = cell_next == 2 ? 0 : cell_next + 1;
+    if (s + 1 < nslab) loader.fetch(p, tid, s + 1, raw);
+    const float na = __uint_as_float(nrm[cell][0]), nb = __uint_as_float(nrm[cell][1]);
+    if (tid < 2) nrm[cell_clear][tid] = 0u;  // read during the previous slab, filled during the next
+    // ||x|| ||w|| / 2^(e_max+1), rounded up generously (the norms carry rounding errors near 2^-20)
+    const float grow = sqrtf(na * nb) * 1.01f;
+    bool fast = __all_sync(0xFFFFFFFFu, u + grow < 0.999f);
+    if (!fast && u > 0.0f) {  // the carried bound may just be loose: measure |acc1|
+      float mx = 0.0f;
+#pragma unroll
+      for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < PN; ++j) {
+          float lo, hi;
+          unpack2(acc1[i][j], lo, hi);
+          mx = fmaxf(mx, fmaxf(fabsf(lo), fabsf(hi)));
+        }
+      u = mx * p.inv_top;
+      fast = __all_sync(0xFFFFFFFFu, u + grow < 0.999f);
+    }
+    if (fast) slab_body(buf, std::false_type());
+    else slab_body(buf, std::true_type());
+    u = fminf(u + grow, 1.0f);
+    if (CHUNKED) {
+      if (++slabs_in_chunk == p.chunk_slabs) {
+        close_chunk();
+        slabs_in_chunk = 0;
+        u = 0.0f;
+      }
+    }
+    if (s + 1 < nslab) decode_store(raw, buf ^ 1, cell_next);
+    __syncthreads();
+    cell = cell_next;
+  }
+  if (CHUNKED && slabs_in_chunk > 0) close_chunk();
+
+  // ---- epilogue: back to real values, +0 for every zero, scales and bias in binary32
+  const bool vec_store = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0);
+#pragma unroll
+  for (int i = 0; i < TM; ++i) {
+    const int64_t m = m0 + (i / 4) * (BM / 2) + ty * 4 + (i % 4);
+    if (m >= p.M) continue;
+    const float sa = p.sa[p.sa_per_row ? m : 0];
+#pragma unroll
+    for (int h = 0; h < TN / 4; ++h) {
+      const int64_t n = n0 + h * (BN / 2) + tx * 4;
+      float o[4];
+#pragma unroll
+      for (int jp = 0; jp < 2; ++jp) {
+        const u64 sv = CHUNKED ? acc2[CHUNKED ? i : 0][CHUNKED ? h * 2 + jp : 0] : acc1[i][h * 2 + jp];
+        unpack2(sv, o[jp * 2], o[jp * 2 + 1]);
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float y = __fmul_rn(__fmul_rn(o[j], p.un1), p.un2);
+        o[j] = (y == 0.0f) ? 0.0f : y;
+      }
+      if (n + 3 < p.N && vec_store) {
+        float4 v;
+        float* ov = &v.x;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float sb = p.sb[p.sb_per_col ? n + j : 0];
+          float r = __fmul_rn(__fmul_rn(o[j], sa), sb);
+          if (p.bias) r = __fadd_rn(r, p.bias[n + j]);
+          ov[j] = r;
+        }
+        *reinterpret_cast<float4*>(p.out + m * p.N + n) = v;
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (n + j < p.N) {
+            const float sb = p.sb[p.sb_per_col ? n + j : 0];
+            float r = __fmul_rn(__fmul_rn(o[j], sa), sb);
+            if (p.bias) r = __fadd_rn(r, p.bias[n + j]);
+            p.out[m * p.N + n + j] = r;
+          }
+        }
+      }
+    }
+  }
+}
+
+template <int BM, int BN>
+constexpr size_t packed_smem_bytes() {
+  return sizeof(float2) * 2 * BK * BM + sizeof(float) * 2 * BK * BN + sizeof(unsigned) * 6;
 }
 
 // Launch entry of one (quantiser mode, order mode) family; defined once per translation unit.
