@@ -15,7 +15,6 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
 import sys
 import threading
 import time
@@ -32,12 +31,19 @@ WORKLOAD = "resnet18_fwd_conv_stack_b32_224_m7e4_chunk16"
 BATCH = 32
 CONFIG_ID = 2
 
-# ALU roofline constants for sm_100: per SM and clock, 128 lanes can be issued and the integer/logic/min-max
-# pipe executes 64 lanes; the fast floor path needs 2 instructions of that pipe per emulated MAC
-# (mantissa mask and magnitude clamp).
+# ALU roofline for sm_100.  Per SM and clock 4 schedulers issue one warp instruction each (128 lanes), the
+# FP32 pipe retires 128 lanes and the integer/logic pipe 64.  The packed floor path needs, per emulated MAC,
+# half an FMUL2 and half an FFMA2 (one FP32 lane-op each) and one LOP3 (the mantissa mask), i.e. 2 issue
+# slots, 2 FP32 lane-ops and 1 logic lane-op: all three limits coincide at 2 clocks per warp-MAC per
+# scheduler.  The chunked order adds, per chunk of `chunk` MACs, one packed add, two masks and two clamps
+# per output pair: (0.5 + 1 + 1) issue slots per output.
 ISSUE_LANES_PER_SM_CLK = 128
-ALU_PIPE_LANES_PER_SM_CLK = 64
-ALU_PIPE_INSTR_PER_MAC = 2.0
+ISSUE_SLOTS_PER_MAC_LEVEL1 = 2.0
+ISSUE_SLOTS_PER_CHUNK_CLOSE = 2.5
+
+
+def issue_slots_per_mac(order_chunked: bool, chunk: int) -> float:
+    return ISSUE_SLOTS_PER_MAC_LEVEL1 + (ISSUE_SLOTS_PER_CHUNK_CLOSE / chunk if order_chunked else 0.0)
 
 
 def parse_args():
@@ -54,35 +60,55 @@ def parse_args():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock and throttle reasons through NVML (read-only queries) while the timed region runs."""
+
+    REASONS = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+               "hw_power_brake_slowdown": 0x80}
 
     def __init__(self, index):
         self.index = index
         self.samples = []
+        self.power = []
         self.reasons = set()
         self.max_mhz = None
         self._stop = threading.Event()
         self._thread = None
+        self._nvml = None
+        self._handle = None
+
+    def _open(self):
+        import pynvml
+        pynvml.nvmlInit()
+        self._nvml = pynvml
+        # NVML numbers devices by PCI order, CUDA possibly by a CUDA_VISIBLE_DEVICES subset: go through the UUID
+        uuid = torch.cuda.get_device_properties(self.index).uuid
+        try:
+            self._handle = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+        except Exception:
+            self._handle = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+        self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._handle, pynvml.NVML_CLOCK_SM))
 
     def _run(self):
-        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        n = self._nvml
         while not self._stop.is_set():
             try:
-                out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={q}",
-                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
-                f = [x.strip() for x in out.strip().split(",")]
-                self.samples.append(float(f[0]))
-                self.max_mhz = float(f[1])
-                for n, v in zip(names, f[2:]):
-                    if v.lower().startswith("active"):
-                        self.reasons.add(n)
+                self.samples.append(float(n.nvmlDeviceGetClockInfo(self._handle, n.NVML_CLOCK_SM)))
+                self.power.append(n.nvmlDeviceGetPowerUsage(self._handle) / 1000.0)
+                mask = n.nvmlDeviceGetCurrentClocksEventReasons(self._handle) if hasattr(
+                    n, "nvmlDeviceGetCurrentClocksEventReasons") else n.nvmlDeviceGetCurrentClocksThrottleReasons(self._handle)
+                for name, bit in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
             except Exception:
                 pass
-            self._stop.wait(0.05)
+            self._stop.wait(0.002)
 
     def start(self):
+        try:
+            self._open()
+        except Exception:
+            self._nvml = None
+            return
         self._thread = threading.Thread(target=self._run, daemon=True)
         self._thread.start()
 
@@ -91,8 +117,9 @@ class ClockSampler:
         if self._thread:
             self._thread.join(timeout=10)
         med = statistics.median(self.samples) if self.samples else None
-        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+        return {"sm_mhz": med, "sm_min_mhz": min(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "power_w_max": max(self.power) if self.power else None,
+                "samples": len(self.samples), "source": "nvml"}
 
 
 def formats():
@@ -283,17 +310,21 @@ def main():
         e["launches"] += 1
     dom_key, dom = max(by_kernel.items(), key=lambda kv: kv[1]["ms"])
     sm_count = torch.cuda.get_device_properties(device).multi_processor_count
-    mhz = clocks["sm_mhz"] or clocks["sm_max_mhz"] or 1965.0
-    alu_pipe_bound = sm_count * ALU_PIPE_LANES_PER_SM_CLK * mhz * 1e6 / ALU_PIPE_INSTR_PER_MAC / 1e9
+    max_mhz = clocks["sm_max_mhz"] or 1965.0
+    mhz = clocks["sm_mhz"] or max_mhz
+    slots = issue_slots_per_mac(True, 16)
+    peak = sm_count * ISSUE_LANES_PER_SM_CLK * max_mhz * 1e6 / slots / 1e9
     achieved = dom["macs"] / (dom["ms"] * 1e-3) / 1e9
     roofline = {
-        "bound": "alu", "achieved": achieved, "peak": alu_pipe_bound, "unit": UNIT, "frac": achieved / alu_pipe_bound,
+        "bound": "alu", "achieved": achieved, "peak": peak, "unit": UNIT, "frac": achieved / peak,
         "traffic": None,
         "kernel": dom_key, "kernel_launches_per_step": dom["launches"], "kernel_ms_per_step": dom["ms"],
         "kernel_share_of_step": dom["ms"] / sum(per_call_ms),
-        "peak_derivation": f"{sm_count} SMs x {ALU_PIPE_LANES_PER_SM_CLK} integer/logic lanes per clock x {mhz:.0f} MHz "
-                           f"(median sampled) / {ALU_PIPE_INSTR_PER_MAC:g} such instructions per emulated MAC",
-        "whole_step_frac_of_peak": (step_macs / (sum(per_call_ms) * 1e-3) / 1e9) / alu_pipe_bound,
+        "peak_derivation": f"{sm_count} SMs x {ISSUE_LANES_PER_SM_CLK} lanes issued per clock x {max_mhz:.0f} MHz "
+                           f"(clocks.max.sm) / {slots:g} issue slots per emulated MAC (0.5 FMUL2 + 0.5 FFMA2 + 1 LOP3, "
+                           f"plus 2.5 per output per chunk of 16); the FP32 and logic pipes give the same limit",
+        "frac_at_sampled_clock": achieved / (peak * mhz / max_mhz),
+        "whole_step_frac_of_peak": (step_macs / (sum(per_call_ms) * 1e-3) / 1e9) / peak,
     }
 
     # ---- end to end through the host-buffer C entry points
