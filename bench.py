@@ -30,6 +30,8 @@ UNIT = "GMAC/s"
 WORKLOAD = "resnet18_fwd_conv_stack_b32_224_m7e4_chunk16"
 BATCH = 32
 CONFIG_ID = 2
+RUN_ORDER = 1        # ORDER_CHUNKED, the paper's order; a single-GEMM workload may ask for the sequential order
+GEMM_CASE = None     # (M, N, K) when --workload gemm:MxNxK[:seq|chunk] replaces the network
 
 # ALU roofline for sm_100.  Per SM and clock 4 schedulers issue one warp instruction each (128 lanes), the
 # FP32 pipe retires 128 lanes and the integer/logic pipe 64.  The packed floor path needs, per emulated MAC,
@@ -49,9 +51,12 @@ def issue_slots_per_mac(order_chunked: bool, chunk: int) -> float:
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet18",
+                    help="resnet18 (default, the benchmark) or gemm:MxNxK[:seq|chunk], one LBA GEMM on Gaussian "
+                         "operands (used for kernel profiles)")
     ap.add_argument("--cpu-baseline-macs", type=float, default=1.5e9,
                     help="size of the oracle sample timed for cpu_baseline (emulated MACs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -128,8 +133,14 @@ def formats():
 
 
 def build_calls(device):
-    from paper_2401_14110_b200 import binding as lba, workloads, ORDER_CHUNKED
+    from paper_2401_14110_b200 import binding as lba, synth, workloads, ORDER_CHUNKED
     prod, acc = formats()
+    if GEMM_CASE is not None:
+        m, n, k = GEMM_CASE
+        a, sa, b, sb = synth.gemm_case(m, n, k, config=5)
+        c = workloads.LbaCall("gemm", "gemm", a.to(device), b.to(device), sa.to(device), sb.to(device))
+        c.out = torch.empty((m, n), dtype=torch.float32, device=device)
+        return [c]
 
     def conv_fn(x, w, sx, sw, stride, pad):
         return lba.lba_conv2d(x, w, sx, sw, None, stride, pad, prod, acc, ORDER_CHUNKED, 16)
@@ -145,7 +156,8 @@ def build_calls(device):
 
 
 def run_step(calls, events=None):
-    from paper_2401_14110_b200 import binding as lba, ORDER_CHUNKED
+    from paper_2401_14110_b200 import binding as lba
+    ORDER_CHUNKED = RUN_ORDER
     prod, acc = formats()
     for i, c in enumerate(calls):
         if events is not None:
@@ -159,7 +171,8 @@ def run_step(calls, events=None):
 
 
 def describe(c):
-    from paper_2401_14110_b200 import binding as lba, ORDER_CHUNKED
+    from paper_2401_14110_b200 import binding as lba
+    ORDER_CHUNKED = RUN_ORDER
     prod, acc = formats()
     m, n, k = c.gemm_shape
     vec = (c.x.shape[-1] % 16 == 0) if c.kind == "conv" else (k % 16 == 0)
@@ -169,9 +182,10 @@ def describe(c):
 def cpu_baseline(calls, target_macs):
     """Time the oracle, as it stands, on a bounded sample: seeded 16x16 output tiles of several layers."""
     from oracle import lba_oracle as orc
-    from paper_2401_14110_b200 import synth, ORDER_CHUNKED
+    from paper_2401_14110_b200 import synth
+    ORDER_CHUNKED = RUN_ORDER
     prod, acc = formats()
-    picks = [c for c in calls if c.kind == "conv"][1::4] + [calls[0]]
+    picks = ([c for c in calls if c.kind == "conv"][1::4] + [calls[0]]) if GEMM_CASE is None else calls
     per_layer = target_macs / len(picks)
     jobs = []
     for i, c in enumerate(picks):
@@ -184,8 +198,12 @@ def cpu_baseline(calls, target_macs):
     t0 = time.perf_counter()
     macs = 0
     for c, x, w, sx, sw, ms, ns, k in jobs:
-        orc.conv2d_points(x, w, sx, sw, None, c.stride, c.pad, prod.as_tuple(), acc.as_tuple(), ORDER_CHUNKED, 16,
-                          ms, ns, nthreads=cores)
+        if c.kind == "conv":
+            orc.conv2d_points(x, w, sx, sw, None, c.stride, c.pad, prod.as_tuple(), acc.as_tuple(), ORDER_CHUNKED, 16,
+                              ms, ns, nthreads=cores)
+        else:
+            orc.gemm_points(x, w, sx, sw, None, prod.as_tuple(), acc.as_tuple(), ORDER_CHUNKED, 16, ms, ns,
+                            nthreads=cores)
         macs += len(ms) * k
     dt = time.perf_counter() - t0
     return {"value": macs / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
@@ -231,7 +249,7 @@ def reference_arm(args):
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "int128 exact dyadic (CPU)", "data": "synthetic",
+        "vs_baseline": None, "dtype": "int128", "data": "synthetic",
         "config": {"workload": WORKLOAD, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -239,7 +257,15 @@ def reference_arm(args):
 
 
 def main():
+    global WORKLOAD, RUN_ORDER, GEMM_CASE
     args = parse_args()
+    if args.workload.startswith("gemm:"):
+        parts = args.workload.split(":")
+        GEMM_CASE = tuple(int(v) for v in parts[1].lower().split("x"))
+        RUN_ORDER = 0 if (len(parts) > 2 and parts[2].startswith("seq")) else 1
+        WORKLOAD = "single_lba_gemm_%dx%dx%d_m7e4_%s" % (GEMM_CASE + ("sequential" if RUN_ORDER == 0 else "chunk16",))
+    elif args.workload != "resnet18":
+        raise SystemExit("unknown --workload")
     if args.impl == "reference":
         reference_arm(args)
         return
@@ -255,7 +281,8 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
 
-    from paper_2401_14110_b200 import binding as lba, ORDER_CHUNKED
+    from paper_2401_14110_b200 import binding as lba
+    ORDER_CHUNKED = RUN_ORDER
     lba.load_library()
     prod, acc = formats()
     calls = build_calls(device)
@@ -312,7 +339,7 @@ def main():
     sm_count = torch.cuda.get_device_properties(device).multi_processor_count
     max_mhz = clocks["sm_max_mhz"] or 1965.0
     mhz = clocks["sm_mhz"] or max_mhz
-    slots = issue_slots_per_mac(True, 16)
+    slots = issue_slots_per_mac(RUN_ORDER == 1, 16)
     peak = sm_count * ISSUE_LANES_PER_SM_CLK * max_mhz * 1e6 / slots / 1e9
     achieved = dom["macs"] / (dom["ms"] * 1e-3) / 1e9
     roofline = {
@@ -381,11 +408,11 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "fp8_e4m3 in, 12-bit M7E4 accumulator emulated in f32 registers, f32 out",
+            "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
             "config": {"workload": WORKLOAD, "batch_per_gpu": BATCH, "lba_calls_per_step": launches_per_step,
                        "macs_per_step_per_gpu": step_macs, "prod_fmt": list(prod.as_tuple()),
-                       "acc_fmt": list(acc.as_tuple()), "order": "chunked", "chunk": 16,
+                       "acc_fmt": list(acc.as_tuple()), "order": "chunked" if RUN_ORDER == 1 else "sequential", "chunk": 16,
                        "l2": f"no flush: each step streams {working_set / 1e6:.0f} MB of distinct operands and "
                              f"outputs, larger than the 126 MB L2",
                        "parallelism": f"dp{world} (batch sharded, weights replicated, no collective)"},
