@@ -68,7 +68,8 @@ enum {
   LBA_ERR_ORDER = -4,     /* unknown order, or chunk < 1 in chunked order                    */
   LBA_ERR_SCALE_LEN = -5, /* a scale length that is neither 1 nor the matching dimension     */
   LBA_ERR_CUDA = -6,      /* a CUDA call failed; see lba_last_cuda_error                     */
-  LBA_ERR_WORKSPACE = -7  /* host-buffer entry points: workspace NULL, too small, misaligned */
+  LBA_ERR_WORKSPACE = -7, /* host-buffer entry points: workspace NULL, too small, misaligned */
+  LBA_ERR_STATIC_LIMIT = -8 /* lba_gemm_host_static: the problem needs more than LBA_STATIC_WORKSPACE_BYTES */
 };
 
 /* GEMM  out[m][n] = epilogue( dot(A[m][:], B[n][:]) ), i.e. Y = X W^T with x_i = X_mi,
@@ -121,6 +122,34 @@ int lba_conv2d_host(const uint8_t* x, const uint8_t* w, const float* scale_x, in
                     int C_out, int KH, int KW, int stride_h, int stride_w, int pad_h, int pad_w,
                     const lba_fmt* prod_fmt, const lba_fmt* acc_fmt, int order, int chunk, float* out,
                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* lba_gemm_host for callers that must not allocate device memory.  (No counterpart in the paper: it
+ * is a packaging variant of lba_gemm_host, computing exactly the same result.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a region whose device memory
+ * is budgeted and handed out up front (an inference server's arena, a plug-in that was given no
+ * allocator), in a callback or a latency-critical loop where an allocation would synchronise the
+ * device, or after start-up in a process that has promised not to grow its footprint.  lba_gemm_host
+ * asks such a caller for a device workspace it has no way to obtain; this entry point brings its own.
+ *
+ * The workspace is a fixed array of LBA_STATIC_WORKSPACE_BYTES bytes that is part of the library
+ * image: every GPU on which the library is loaded holds that much memory from load until the process
+ * exits, whether or not this function is ever called.  Arguments are those of lba_gemm_host without
+ * the workspace pair; A, B, scales, bias and out are HOST buffers, copied on `stream`.
+ *   - A problem with lba_gemm_host_workspace_bytes(...) > LBA_STATIC_WORKSPACE_BYTES is refused with
+ *     LBA_ERR_STATIC_LIMIT and nothing is enqueued (roughly: M*K + N*K + 4*M*N must fit in 8 MiB).
+ *   - The first call on each device looks up the array's device address (once, with that device
+ *     current) and keeps it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left there.
+ *     Nothing in it has to start at zero: each call overwrites the operand areas it reads and the
+ *     kernel writes every output element before it is copied back.  Two calls whose work overlaps on
+ *     the GPU (different streams, or different host threads) race on the array: serialise them.
+ *   - No cudaMalloc, cudaFree or other allocating call is made, on the first call or later. */
+#define LBA_STATIC_WORKSPACE_BYTES (8u << 20)
+int lba_gemm_host_static(const uint8_t* A, const uint8_t* B, const float* scale_a, int scale_a_len,
+                         const float* scale_b, int scale_b_len, const float* bias, int64_t M, int64_t N, int64_t K,
+                         const lba_fmt* prod_fmt, const lba_fmt* acc_fmt, int order, int chunk, float* out,
+                         void* stream);
 
 /* Debug helper for the NaN-code precondition: adds to *count (device, uint64, caller zeroes
  * it) the number of bytes among codes[0..n) equal to 0x7F or 0xFF. */

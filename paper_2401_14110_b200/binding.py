@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liblba.so")
 
 EXPORTS = ["lba_gemm", "lba_conv2d", "lba_gemm_host_workspace_bytes", "lba_gemm_host",
-           "lba_conv2d_host_workspace_bytes", "lba_conv2d_host", "lba_count_nan_codes", "lba_describe_plan",
+           "lba_conv2d_host_workspace_bytes", "lba_conv2d_host", "lba_gemm_host_static", "lba_count_nan_codes", "lba_describe_plan",
            "lba_set_tile_override", "lba_status_string", "lba_last_cuda_error", "lba_version"]
 
 
@@ -53,6 +53,7 @@ def load_library():
                  C.c_int64, C.POINTER(_Fmt), C.POINTER(_Fmt), C.c_int, C.c_int, C.c_void_p]
     lib.lba_gemm.argtypes = gemm_args + [C.c_void_p]
     lib.lba_gemm_host.argtypes = gemm_args + [C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.lba_gemm_host_static.argtypes = gemm_args + [C.c_void_p]
     conv_args = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p] + [C.c_int] * 11 + \
         [C.POINTER(_Fmt), C.POINTER(_Fmt), C.c_int, C.c_int, C.c_void_p]
     lib.lba_conv2d.argtypes = conv_args + [C.c_void_p]
@@ -157,6 +158,25 @@ def lba_gemm_host(A, B, scale_a, scale_b, bias, prod_fmt, acc_fmt, order, chunk,
                              _host(bias, torch.float32, "bias"), M, N, K, C.byref(pf), C.byref(af), order, chunk,
                              _host(out, torch.float32, "out"), _dev(workspace, torch.uint8, "workspace"),
                              workspace.numel(), _stream(stream)))
+    return out
+
+
+STATIC_WORKSPACE_BYTES = 8 << 20   # LBA_STATIC_WORKSPACE_BYTES in lba.h
+
+
+def lba_gemm_host_static(A, B, scale_a, scale_b, bias, prod_fmt, acc_fmt, order, chunk, out, stream=None):
+    """``lba_gemm_host`` for callers that cannot allocate device memory: CPU tensors in, CPU ``out``, and the
+    device workspace is an 8 MiB array built into the library (shared by all calls on a device, so calls must
+    not overlap on the GPU).  Larger problems raise ``LbaError`` with status -8.  No tensor is created here."""
+    lib = load_library()
+    M, K = A.shape
+    N, _ = B.shape
+    pf, af = _fmt(prod_fmt), _fmt(acc_fmt)
+    _check(lib.lba_gemm_host_static(_host(A, torch.uint8, "A"), _host(B, torch.uint8, "B"),
+                                    _host(scale_a, torch.float32, "scale_a"), scale_a.numel(),
+                                    _host(scale_b, torch.float32, "scale_b"), scale_b.numel(),
+                                    _host(bias, torch.float32, "bias"), M, N, K, C.byref(pf), C.byref(af), order,
+                                    chunk, _host(out, torch.float32, "out"), _stream(stream)))
     return out
 
 

@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "../../include/lba.h"
 #include "lba_kernel.cuh"
@@ -299,6 +300,7 @@ const char* lba_status_string(int status) {
     case LBA_ERR_SCALE_LEN: return "scale length must be 1 or the matching dimension";
     case LBA_ERR_CUDA: return "a CUDA call failed (see lba_last_cuda_error)";
     case LBA_ERR_WORKSPACE: return "workspace missing, too small or misaligned";
+    case LBA_ERR_STATIC_LIMIT: return "problem too large for the built-in workspace of lba_gemm_host_static (LBA_STATIC_WORKSPACE_BYTES)";
     default: return "unknown status";
   }
 }
@@ -478,3 +480,53 @@ int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, 
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------ lba_gemm_host without allocation
+// The device workspace of lba_gemm_host, as an array inside the library image.  In host code the
+// name `g_static_workspace` is only a handle for the runtime, not a device address: the address the
+// copies and the kernel need comes from cudaGetSymbolAddress, asked once per device.
+namespace {
+
+static __device__ __align__(256) unsigned char g_static_workspace[LBA_STATIC_WORKSPACE_BYTES];
+
+constexpr int kMaxDevices = 64;
+void* g_static_workspace_addr[kMaxDevices] = {};
+std::mutex g_static_workspace_mutex;
+
+// Device address of the array on the current device; looked up on the first call there.
+int static_workspace(void** addr) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= kMaxDevices) return cuda_fail(cudaErrorInvalidDevice);
+  std::lock_guard<std::mutex> lock(g_static_workspace_mutex);
+  if (!g_static_workspace_addr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_workspace);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (!p) return cuda_fail(cudaErrorInvalidSymbol);
+    g_static_workspace_addr[dev] = p;
+  }
+  *addr = g_static_workspace_addr[dev];
+  return LBA_OK;
+}
+
+}  // namespace
+
+extern "C" int lba_gemm_host_static(const uint8_t* A, const uint8_t* B, const float* scale_a, int scale_a_len,
+                                    const float* scale_b, int scale_b_len, const float* bias, int64_t M, int64_t N,
+                                    int64_t K, const lba_fmt* prod_fmt, const lba_fmt* acc_fmt, int order, int chunk,
+                                    float* out, void* stream) {
+  if (M < 0 || N < 0 || K < 0) return LBA_ERR_SHAPE;
+  if (scale_a_len < 0 || scale_b_len < 0) return LBA_ERR_SCALE_LEN;
+  // refuse before touching the device: sizes are compared in double first so that a huge shape cannot wrap size_t
+  const double rough = (double)M * (double)K + (double)N * (double)K + 4.0 * (double)M * (double)N;
+  if (rough > (double)LBA_STATIC_WORKSPACE_BYTES) return LBA_ERR_STATIC_LIMIT;
+  const size_t need = lba_gemm_host_workspace_bytes(M, N, K, scale_a_len, scale_b_len, bias != nullptr);
+  if (need > (size_t)LBA_STATIC_WORKSPACE_BYTES) return LBA_ERR_STATIC_LIMIT;
+  void* ws = nullptr;
+  const int st = static_workspace(&ws);
+  if (st != LBA_OK) return st;
+  return lba_gemm_host(A, B, scale_a, scale_a_len, scale_b, scale_b_len, bias, M, N, K, prod_fmt, acc_fmt, order, chunk,
+                       out, ws, (size_t)LBA_STATIC_WORKSPACE_BYTES, stream);
+}
