@@ -14,6 +14,7 @@ namespace lba {
 // one definition per (QM, ORD), in the lba_fam_*.cu translation units
 #define LBA_DECL(QM, ORD) template <> cudaError_t launch_family<QM, ORD>(int, int, const Problem&, cudaStream_t);
 LBA_DECL(QM_FLOOR_FAST, ORD_SEQ) LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK_SLAB) LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK_ANY)
+LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK16)
 LBA_DECL(QM_FLOOR_FULL, ORD_SEQ) LBA_DECL(QM_FLOOR_FULL, ORD_CHUNK_SLAB) LBA_DECL(QM_FLOOR_FULL, ORD_CHUNK_ANY)
 LBA_DECL(QM_RNE_FULL, ORD_SEQ) LBA_DECL(QM_RNE_FULL, ORD_CHUNK_SLAB) LBA_DECL(QM_RNE_FULL, ORD_CHUNK_ANY)
 LBA_DECL(QM_RNE_WIDE, ORD_SEQ) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_SLAB) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_ANY)
@@ -30,18 +31,20 @@ int cuda_fail(cudaError_t e) {
 }
 
 const LaunchFn kLaunch[QM_COUNT][ORD_COUNT] = {
+    // last column: chunk == 16 has a kernel of its own only for the fast floor quantiser (the plan never
+    // selects it for the others; their entries repeat the general chunk-of-slabs family)
     {launch_family<QM_FLOOR_FAST, ORD_SEQ>, launch_family<QM_FLOOR_FAST, ORD_CHUNK_SLAB>,
-     launch_family<QM_FLOOR_FAST, ORD_CHUNK_ANY>},
+     launch_family<QM_FLOOR_FAST, ORD_CHUNK_ANY>, launch_family<QM_FLOOR_FAST, ORD_CHUNK16>},
     {launch_family<QM_FLOOR_FULL, ORD_SEQ>, launch_family<QM_FLOOR_FULL, ORD_CHUNK_SLAB>,
-     launch_family<QM_FLOOR_FULL, ORD_CHUNK_ANY>},
+     launch_family<QM_FLOOR_FULL, ORD_CHUNK_ANY>, launch_family<QM_FLOOR_FULL, ORD_CHUNK_SLAB>},
     {launch_family<QM_RNE_FULL, ORD_SEQ>, launch_family<QM_RNE_FULL, ORD_CHUNK_SLAB>,
-     launch_family<QM_RNE_FULL, ORD_CHUNK_ANY>},
+     launch_family<QM_RNE_FULL, ORD_CHUNK_ANY>, launch_family<QM_RNE_FULL, ORD_CHUNK_SLAB>},
     {launch_family<QM_RNE_WIDE, ORD_SEQ>, launch_family<QM_RNE_WIDE, ORD_CHUNK_SLAB>,
-     launch_family<QM_RNE_WIDE, ORD_CHUNK_ANY>},
+     launch_family<QM_RNE_WIDE, ORD_CHUNK_ANY>, launch_family<QM_RNE_WIDE, ORD_CHUNK_SLAB>},
 };
 
 const char* const kQmName[QM_COUNT] = {"floor_fast", "floor_full", "rne_full", "rne_wide"};
-const char* const kOrdName[ORD_COUNT] = {"seq", "chunk_slab", "chunk_any"};
+const char* const kOrdName[ORD_COUNT] = {"seq", "chunk_slab", "chunk_any", "chunk16"};
 const char* const kLdName[LD_COUNT] = {"gemm_vec", "conv_vec", "any"};
 
 // Largest |x*w| of two E4M3 values and the grid every product lies on.
@@ -169,7 +172,7 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
   if (order == LBA_ORDER_SEQUENTIAL || (int64_t)chunk >= K) {
     pl->ord = ORD_SEQ;  // a single chunk: the second hierarchy adds it to 0, which changes nothing
   } else if (chunk % BK == 0) {
-    pl->ord = ORD_CHUNK_SLAB;
+    pl->ord = (chunk == BK && pl->qm == QM_FLOOR_FAST) ? ORD_CHUNK16 : ORD_CHUNK_SLAB;
     pl->chunk_slabs = chunk / BK;
   } else {
     pl->ord = ORD_CHUNK_ANY;

@@ -33,7 +33,8 @@
 namespace lba {
 
 enum QMode { QM_FLOOR_FAST = 0, QM_FLOOR_FULL = 1, QM_RNE_FULL = 2, QM_RNE_WIDE = 3, QM_COUNT = 4 };
-enum OrdMode { ORD_SEQ = 0, ORD_CHUNK_SLAB = 1, ORD_CHUNK_ANY = 2, ORD_COUNT = 3 };
+// ORD_CHUNK16: chunk == BK, the paper's chunk size; only the packed floor kernel specialises it
+enum OrdMode { ORD_SEQ = 0, ORD_CHUNK_SLAB = 1, ORD_CHUNK_ANY = 2, ORD_CHUNK16 = 3, ORD_COUNT = 4 };
 enum LoadMode { LD_GEMM_VEC = 0, LD_CONV_VEC = 1, LD_ANY = 2, LD_COUNT = 3 };
 
 constexpr int BK = 16;  // bytes of K per row per slab = one 128-bit load = one paper-sized chunk
@@ -462,6 +463,11 @@ __device__ __forceinline__ u64 fma2_rz_ftz(u64 a, u64 b, u64 c) {
   asm("fma.rz.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
   return d;
 }
+__device__ __forceinline__ u64 mul2_rz_ftz(u64 a, u64 b) {
+  u64 d;
+  asm("mul.rz.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 __device__ __forceinline__ u64 add2_rz_ftz(u64 a, u64 b) {
   u64 d;
   asm("add.rz.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
@@ -486,8 +492,9 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
   constexpr int ROWS = BM + BN;
   constexpr int LPT = (ROWS + NT - 1) / NT;
   constexpr int PN = TN / 2;  // register pairs per micro-tile row
-  constexpr bool CHUNKED = ORD == ORD_CHUNK_SLAB;
-  static_assert(ORD == ORD_SEQ || ORD == ORD_CHUNK_SLAB, "order");
+  constexpr bool CH16 = ORD == ORD_CHUNK16;  // every slab is exactly one chunk
+  constexpr bool CHUNKED = ORD == ORD_CHUNK_SLAB || CH16;
+  static_assert(ORD == ORD_SEQ || ORD == ORD_CHUNK_SLAB || ORD == ORD_CHUNK16, "order");
   static_assert(TM == 4 || TM == 8, "micro-tile rows");
   static_assert(TN == 4 || TN == 8, "micro-tile cols");
   static_assert(BM % 32 == 0 && BN % 32 == 0, "a warp loads rows of one operand only");
@@ -557,10 +564,13 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
   const uint32_t mask = p.qa.mask;
   const float sat = p.qa.sat;
 
-  // one slab of 16 k-steps; CLAMP selects whether the magnitude clamp of Eq. 2 is applied
+  // one slab of 16 k-steps; CLAMP selects whether the magnitude clamp of Eq. 2 is applied.  The clamped
+  // variant is the rare one and stays a rolled loop.  In chunk-16 order the slab starts a chunk: its first
+  // step adds to zero, which is a plain (exact) scaling of the product, so the sums need no clearing.
   auto slab_body = [&](int buf, auto clamp_tag) {
     constexpr bool CLAMP = decltype(clamp_tag)::value;
-#pragma unroll KUNROLL
+    constexpr int UNR = CLAMP ? 1 : KUNROLL;
+#pragma unroll UNR
     for (int kk = 0; kk < BK; ++kk) {
       u64 a2[TM], b2[PN];
 #pragma unroll
@@ -578,7 +588,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
       for (int i = 0; i < TM; ++i)
 #pragma unroll
         for (int j = 0; j < PN; ++j) {
-          const u64 t = fma2_rz_ftz(mul2_ftz(a2[i], b2[j]), cc2, acc1[i][j]);
+          const u64 pr = mul2_ftz(a2[i], b2[j]);
+          const u64 t = (CH16 && kk == 0) ? mul2_rz_ftz(pr, cc2) : fma2_rz_ftz(pr, cc2, acc1[i][j]);
           float lo, hi;
           unpack2(t, lo, hi);
           lo = and_bits(lo, mask);
@@ -592,7 +603,10 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
     }
   };
 
-  auto close_chunk = [&]() {  // second hierarchy: T <- Q_acc(C + T), C <- 0 (always clamped: once per chunk)
+  // second hierarchy: T <- Q_acc(C + T), C <- 0.  With CLAMP the largest |T| is returned as well.
+  auto close_chunk = [&](auto clamp_tag) -> float {
+    constexpr bool CLAMP = decltype(clamp_tag)::value;
+    float mx = 0.0f;
 #pragma unroll
     for (int i = 0; i < TM; ++i)
 #pragma unroll
@@ -600,9 +614,17 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
         u64& t2 = acc2[CHUNKED ? i : 0][CHUNKED ? j : 0];
         float lo, hi;
         unpack2(add2_rz_ftz(acc1[i][j], t2), lo, hi);
-        t2 = pack2(clamp_mag(and_bits(lo, mask), sat), clamp_mag(and_bits(hi, mask), sat));
-        acc1[i][j] = 0ull;
+        lo = and_bits(lo, mask);
+        hi = and_bits(hi, mask);
+        if (CLAMP) {
+          lo = clamp_mag(lo, sat);
+          hi = clamp_mag(hi, sat);
+          mx = fmaxf(mx, fmaxf(fabsf(lo), fabsf(hi)));
+        }
+        t2 = pack2(lo, hi);
+        if (!CH16) acc1[i][j] = 0ull;
       }
+    return mx;
   };
 
   if (tid < 6) nrm[tid >> 1][tid & 1] = 0u;
@@ -614,9 +636,10 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
   }
   __syncthreads();
 
-  float u = 0.0f;  // upper bound of max |acc1| of this thread, as a fraction of 2^(e_max + 1)
+  float u = 0.0f;   // upper bound of max |acc1| of this thread, as a fraction of 2^(e_max + 1)
+  float u2 = 0.0f;  // chunk-16 order: the same for the second-level sums
   int slabs_in_chunk = 0;
-  int cell = 0;    // s % 3
+  int cell = 0;     // s % 3
   for (int s = 0; s < nslab; ++s) {
     const int buf = s & 1;
     const int cell_next = cell == 2 ? 0 : cell + 1;
@@ -626,35 +649,48 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
     if (tid < 2) nrm[cell_clear][tid] = 0u;  // read during the previous slab, filled during the next
     // ||x|| ||w|| / 2^(e_max+1), rounded up generously (the norms carry rounding errors near 2^-20)
     const float grow = sqrtf(na * nb) * 1.01f;
-    bool fast = __all_sync(0xFFFFFFFFu, u + grow < 0.999f);
-    if (!fast && u > 0.0f) {  // the carried bound may just be loose: measure |acc1|
-      float mx = 0.0f;
+    if (CH16) {
+      // the chunk starts from zero, so the CTA-wide bound alone decides (same value in every thread)
+      if (grow < 0.999f) slab_body(buf, std::false_type());
+      else slab_body(buf, std::true_type());
+      // |T + C| <= |T| + |C| <= u2 + grow: below 1 the mask alone already respects R_OF
+      if (__all_sync(0xFFFFFFFFu, u2 + grow < 0.999f)) {
+        close_chunk(std::false_type());
+        u2 += grow;
+      } else {
+        u2 = close_chunk(std::true_type()) * p.inv_top;  // clamped, and the bound is refreshed from the sums
+      }
+    } else {
+      bool fast = __all_sync(0xFFFFFFFFu, u + grow < 0.999f);
+      if (!fast && u > 0.0f) {  // the carried bound may just be loose: measure |acc1|
+        float mx = 0.0f;
 #pragma unroll
-      for (int i = 0; i < TM; ++i)
+        for (int i = 0; i < TM; ++i)
 #pragma unroll
-        for (int j = 0; j < PN; ++j) {
-          float lo, hi;
-          unpack2(acc1[i][j], lo, hi);
-          mx = fmaxf(mx, fmaxf(fabsf(lo), fabsf(hi)));
+          for (int j = 0; j < PN; ++j) {
+            float lo, hi;
+            unpack2(acc1[i][j], lo, hi);
+            mx = fmaxf(mx, fmaxf(fabsf(lo), fabsf(hi)));
+          }
+        u = mx * p.inv_top;
+        fast = __all_sync(0xFFFFFFFFu, u + grow < 0.999f);
+      }
+      if (fast) slab_body(buf, std::false_type());
+      else slab_body(buf, std::true_type());
+      u = fminf(u + grow, 1.0f);
+      if (CHUNKED) {
+        if (++slabs_in_chunk == p.chunk_slabs) {
+          close_chunk(std::true_type());
+          slabs_in_chunk = 0;
+          u = 0.0f;
         }
-      u = mx * p.inv_top;
-      fast = __all_sync(0xFFFFFFFFu, u + grow < 0.999f);
-    }
-    if (fast) slab_body(buf, std::false_type());
-    else slab_body(buf, std::true_type());
-    u = fminf(u + grow, 1.0f);
-    if (CHUNKED) {
-      if (++slabs_in_chunk == p.chunk_slabs) {
-        close_chunk();
-        slabs_in_chunk = 0;
-        u = 0.0f;
       }
     }
     if (s + 1 < nslab) decode_store(raw, buf ^ 1, cell_next);
     __syncthreads();
     cell = cell_next;
   }
-  if (CHUNKED && slabs_in_chunk > 0) close_chunk();
+  if (CHUNKED && !CH16 && slabs_in_chunk > 0) close_chunk(std::true_type());
 
   // ---- epilogue: back to real values, +0 for every zero, scales and bias in binary32
   const bool vec_store = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0);

@@ -33,7 +33,7 @@ def test_plan_selection_by_format_and_order():
     p, a = code_domain_formats(7, 4)
     assert "q=floor_fast" in lba.describe_plan(64, 64, 576, p, a, SEQ, 16)
     assert "order=seq" in lba.describe_plan(64, 64, 576, p, a, SEQ, 16)
-    assert "order=chunk_slab" in lba.describe_plan(64, 64, 576, p, a, CHK, 16)
+    assert "order=chunk16" in lba.describe_plan(64, 64, 576, p, a, CHK, 16)
     assert "order=chunk_slab" in lba.describe_plan(64, 64, 576, p, a, CHK, 32)
     assert "order=chunk_any" in lba.describe_plan(64, 64, 576, p, a, CHK, 5)
     assert "order=seq" in lba.describe_plan(64, 64, 576, p, a, CHK, 576)       # one chunk == sequential
