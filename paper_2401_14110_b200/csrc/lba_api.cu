@@ -180,27 +180,29 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
   return LBA_OK;
 }
 
-// Tile choice: the largest tile that still gives every SM work; smaller tiles cost more loads and
-// decodes per MAC, larger ones leave SMs idle on small problems.
-int choose_tile(int64_t M, int64_t N, int ord) {
+// Tile choice.  All CTAs of a launch have the same work and K is never split, so the launch ends when the
+// busiest SM has run its ceil(CTAs / SMs) tiles; larger tiles spend fewer instructions per MAC (eff, measured
+// on B200 with every SM loaded), smaller ones fill the SMs more evenly.  Pick the cheapest by that model.
+bool packed_plan(int qm, int ord) { return qm == QM_FLOOR_FAST && ord != ORD_CHUNK_ANY; }
+
+int choose_tile(int64_t M, int64_t N, int qm, int ord) {
+  (void)qm;
+  (void)ord;
   if (g_tile_override >= 0) return g_tile_override;
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) {
     int v = 0;
     if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
   }
-  // CTAs resident per SM (register-limited) and relative per-MAC efficiency of each tile
-  const int resident[TILE_COUNT] = {1, ord == ORD_SEQ ? 2 : 2, 3, 8};
-  const double eff[TILE_COUNT] = {1.00, 0.97, 0.92, 0.80};
+  const double eff[TILE_COUNT] = {1.00, 0.96, 0.88, 0.87};
   int best = 0;
   double best_cost = 1e300;
   for (int t = 0; t < TILE_COUNT; ++t) {
     const TileInfo ti = tile_info(t);
     const double ctas = (double)((M + ti.bm - 1) / ti.bm) * (double)((N + ti.bn - 1) / ti.bn);
-    const double slots = (double)sms * resident[t];
-    const double waves = std::ceil(ctas / slots);
-    // time ~ waves * (work of the CTAs sharing an SM) / efficiency
-    const double cost = waves * resident[t] * ti.bm * ti.bn / eff[t];
+    const double per_sm = std::ceil(ctas / sms);
+    double cost = per_sm * ti.bm * ti.bn / eff[t];
+    if (t == 0 && per_sm < 2) cost /= 0.85;  // one 8-warp CTA alone does not keep an SM's pipes busy
     if (cost < best_cost) {
       best_cost = cost;
       best = t;
@@ -241,7 +243,7 @@ bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15)
 
 int run(const Problem& p, const Plan& pl, int load, cudaStream_t stream) {
   if (p.M == 0 || p.N == 0) return LBA_OK;
-  const int tile = choose_tile(p.M, p.N, pl.ord);
+  const int tile = choose_tile(p.M, p.N, pl.qm, pl.ord);
   const TileInfo ti = tile_info(tile);
   if ((p.N + ti.bn - 1) / ti.bn > 65535 || (p.M + ti.bm - 1) / ti.bm > 2147483647LL) return LBA_ERR_SHAPE;
   const cudaError_t e = kLaunch[pl.qm][pl.ord](tile, load, p, stream);
@@ -472,7 +474,7 @@ int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, 
   Plan pl;
   const int st = make_plan(prod_fmt, acc_fmt, order, chunk, K, &pl);
   if (st != LBA_OK) return st;
-  const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, pl.ord);
+  const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, pl.qm, pl.ord);
   const TileInfo ti = tile_info(tile);
   const int load = vec_ok ? (is_conv ? LD_CONV_VEC : LD_GEMM_VEC) : LD_ANY;
   if (buf && buf_len)

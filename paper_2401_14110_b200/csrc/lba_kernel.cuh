@@ -485,8 +485,37 @@ __device__ __forceinline__ void e4m3x2_to_f32(uint32_t pair, float& v0, float& v
       : "r"(pair));
 }
 
+// ---- tensor memory as a second register file.  In chunk-16 order the second-level sums T are touched
+// once per 16 k-steps; keeping them in TMEM (each thread owns TM*TN 32-bit columns of its own lane)
+// frees TM*TN registers, which doubles the CTAs an SM can hold for the 8-row micro-tiles.  No MMA is
+// involved: tcgen05.ld / tcgen05.st move 16 columns of a lane to and from registers.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]) : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ u64 pack2u(uint32_t lo, uint32_t hi) {
+  u64 d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
+
+// columns of tensor memory a CTA of the packed kernel allocates (0: second-level sums stay in registers)
+template <int BM, int BN, int TM, int TN, int ORD>
+__host__ __device__ constexpr int packed_tmem_cols() {
+  constexpr int warps = (BM / TM) * (BN / TN) / 32;
+  constexpr int cols = ((warps + 3) / 4) * TM * TN;
+  return (ORD == ORD_CHUNK16 && TM == 8) ? (cols < 32 ? 32 : cols) : 0;
+}
+
+// the 8x8 micro-tile is held to 128 registers (two CTAs of 256 threads per SM) wherever the second-level
+// sums are not in registers
 template <int BM, int BN, int TM, int TN, int ORD, int LD>
-__global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_kernel(const Problem p) {
+__global__ void __launch_bounds__((BM / TM) * (BN / TN), (TM * TN == 64 && ORD != ORD_CHUNK_SLAB) ? 512 / ((BM / TM) * (BN / TN)) : 1)
+    lba_contract_packed_kernel(const Problem p) {
   constexpr int NT = (BM / TM) * (BN / TN);
   constexpr int TX = BN / TN;
   constexpr int ROWS = BM + BN;
@@ -494,6 +523,10 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
   constexpr int PN = TN / 2;  // register pairs per micro-tile row
   constexpr bool CH16 = ORD == ORD_CHUNK16;  // every slab is exactly one chunk
   constexpr bool CHUNKED = ORD == ORD_CHUNK_SLAB || CH16;
+  constexpr int TMEM_COLS = packed_tmem_cols<BM, BN, TM, TN, ORD>();
+  constexpr bool T_IN_TMEM = TMEM_COLS > 0;   // second-level sums in tensor memory
+  constexpr bool T_IN_REGS = CHUNKED && !T_IN_TMEM;
+  static_assert(!T_IN_TMEM || (TM * TN) % 16 == 0, "tensor-memory groups of 16 columns");
   static_assert(ORD == ORD_SEQ || ORD == ORD_CHUNK_SLAB || ORD == ORD_CHUNK16, "order");
   static_assert(TM == 4 || TM == 8, "micro-tile rows");
   static_assert(TN == 4 || TN == 8, "micro-tile cols");
@@ -509,6 +542,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
   // like integers): [slab % 3][0 = A, 1 = B]; three cells so that one can be cleared while the
   // neighbours are read and filled
   unsigned (*nrm)[2] = reinterpret_cast<unsigned (*)[2]>(smem_raw + sizeof(float2) * 2 * BK * BM + sizeof(float) * 2 * BK * BN);
+  unsigned* tmem_slot = reinterpret_cast<unsigned*>(nrm) + 6;  // base address written by tcgen05.alloc
 
   const int tid = threadIdx.x;
   const int tx = tid % TX, ty = tid / TX;
@@ -548,16 +582,16 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
   };
 
   u64 acc1[TM][PN];
-  u64 acc2[CHUNKED ? TM : 1][CHUNKED ? PN : 1];
+  u64 acc2[T_IN_REGS ? TM : 1][T_IN_REGS ? PN : 1];
 #pragma unroll
   for (int i = 0; i < TM; ++i)
 #pragma unroll
     for (int j = 0; j < PN; ++j) acc1[i][j] = 0ull;
-  if (CHUNKED) {
+  if (T_IN_REGS) {
 #pragma unroll
     for (int i = 0; i < TM; ++i)
 #pragma unroll
-      for (int j = 0; j < PN; ++j) acc2[CHUNKED ? i : 0][CHUNKED ? j : 0] = 0ull;
+      for (int j = 0; j < PN; ++j) acc2[T_IN_REGS ? i : 0][T_IN_REGS ? j : 0] = 0ull;
   }
 
   const u64 cc2 = pack2(p.c, p.c);
@@ -611,7 +645,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
     for (int i = 0; i < TM; ++i)
 #pragma unroll
       for (int j = 0; j < PN; ++j) {
-        u64& t2 = acc2[CHUNKED ? i : 0][CHUNKED ? j : 0];
+        u64& t2 = acc2[T_IN_REGS ? i : 0][T_IN_REGS ? j : 0];
         float lo, hi;
         unpack2(add2_rz_ftz(acc1[i][j], t2), lo, hi);
         lo = and_bits(lo, mask);
@@ -627,8 +661,78 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
     return mx;
   };
 
+  // the same with T in tensor memory: 16 columns (16 / TN micro-tile rows) at a time, the next group's
+  // load in flight while the current one is processed.  FINAL leaves the new T in acc1 for the epilogue
+  // instead of storing it back.
+  uint32_t taddr = 0;
+  auto close_chunk_tmem = [&](auto clamp_tag, auto final_tag) -> float {
+    constexpr bool CLAMP = decltype(clamp_tag)::value;
+    constexpr bool FINAL = decltype(final_tag)::value;
+    constexpr int GROUPS = TM * TN / 16;
+    constexpr int ROWS_PER_GROUP = 16 / TN;
+    float mx = 0.0f;
+    uint32_t cur[16], nxt[16];
+    tmem_ld16(taddr, cur);
+#pragma unroll
+    for (int g = 0; g < GROUPS; ++g) {
+      tmem_wait_ld();
+      if (g + 1 < GROUPS) tmem_ld16(taddr + 16 * (g + 1), nxt);
+#pragma unroll
+      for (int r = 0; r < ROWS_PER_GROUP; ++r)
+#pragma unroll
+        for (int j = 0; j < PN; ++j) {
+          const int i = g * ROWS_PER_GROUP + r;
+          const int c = r * TN + 2 * j;
+          float lo, hi;
+          unpack2(add2_rz_ftz(acc1[i][j], pack2u(cur[c], cur[c + 1])), lo, hi);
+          lo = and_bits(lo, mask);
+          hi = and_bits(hi, mask);
+          if (CLAMP) {
+            lo = clamp_mag(lo, sat);
+            hi = clamp_mag(hi, sat);
+            mx = fmaxf(mx, fmaxf(fabsf(lo), fabsf(hi)));
+          }
+          if (FINAL) {
+            acc1[i][j] = pack2(lo, hi);
+          } else {
+            cur[c] = __float_as_uint(lo);
+            cur[c + 1] = __float_as_uint(hi);
+          }
+        }
+      if (!FINAL) tmem_st16(taddr + 16 * g, cur);
+      if (g + 1 < GROUPS) {
+#pragma unroll
+        for (int c = 0; c < 16; ++c) cur[c] = nxt[c];
+      }
+    }
+    if (!FINAL) tmem_wait_st();  // the next close reads these columns again
+    return mx;
+  };
+
   if (tid < 6) nrm[tid >> 1][tid & 1] = 0u;
+  if (T_IN_TMEM) {
+    // one warp allocates for the CTA; tcgen05.alloc returns once the SM has the columns free (CTAs
+    // that hold columns never wait for anything before they release them at the end of the kernel)
+    if (tid < 32) {
+      const uint32_t slot = (uint32_t)__cvta_generic_to_shared(tmem_slot);
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  }
   __syncthreads();
+  if (T_IN_TMEM) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int warp = tid >> 5;
+    // lanes: a warp may touch only the quadrant (warp % 4); warps of the same quadrant take different columns
+    taddr = *tmem_slot + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((warp >> 2) * TM * TN);
+    uint32_t zero[16];
+#pragma unroll
+    for (int c = 0; c < 16; ++c) zero[c] = 0u;
+#pragma unroll
+    for (int g = 0; g < TM * TN / 16; ++g) tmem_st16(taddr + 16 * g, zero);
+    tmem_wait_st();
+  }
   uint4 raw[LPT];
   if (nslab > 0) {
     loader.fetch(p, tid, 0, raw);
@@ -654,11 +758,18 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
       if (grow < 0.999f) slab_body(buf, std::false_type());
       else slab_body(buf, std::true_type());
       // |T + C| <= |T| + |C| <= u2 + grow: below 1 the mask alone already respects R_OF
+      const bool last = T_IN_TMEM && s + 1 == nslab;  // the final T goes to registers for the epilogue
       if (__all_sync(0xFFFFFFFFu, u2 + grow < 0.999f)) {
-        close_chunk(std::false_type());
+        if (!T_IN_TMEM) close_chunk(std::false_type());
+        else if (!last) close_chunk_tmem(std::false_type(), std::false_type());
+        else close_chunk_tmem(std::false_type(), std::true_type());
         u2 += grow;
-      } else {
-        u2 = close_chunk(std::true_type()) * p.inv_top;  // clamped, and the bound is refreshed from the sums
+      } else {  // clamped, and the bound is refreshed from the sums
+        float mx;
+        if (!T_IN_TMEM) mx = close_chunk(std::true_type());
+        else if (!last) mx = close_chunk_tmem(std::true_type(), std::false_type());
+        else mx = close_chunk_tmem(std::true_type(), std::true_type());
+        u2 = mx * p.inv_top;
       }
     } else {
       bool fast = __all_sync(0xFFFFFFFFu, u + grow < 0.999f);
@@ -691,6 +802,13 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
     cell = cell_next;
   }
   if (CHUNKED && !CH16 && slabs_in_chunk > 0) close_chunk(std::true_type());
+  if (T_IN_TMEM) {  // every thread is done with its columns (with K = 0 nothing was ever closed and acc1 is 0)
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (tid < 32) {
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_slot), "r"(TMEM_COLS) : "memory");
+    }
+  }
 
   // ---- epilogue: back to real values, +0 for every zero, scales and bias in binary32
   const bool vec_store = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0);
@@ -705,7 +823,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
       float o[4];
 #pragma unroll
       for (int jp = 0; jp < 2; ++jp) {
-        const u64 sv = CHUNKED ? acc2[CHUNKED ? i : 0][CHUNKED ? h * 2 + jp : 0] : acc1[i][h * 2 + jp];
+        const u64 sv = T_IN_REGS ? acc2[T_IN_REGS ? i : 0][T_IN_REGS ? h * 2 + jp : 0] : acc1[i][h * 2 + jp];
         unpack2(sv, o[jp * 2], o[jp * 2 + 1]);
       }
 #pragma unroll
@@ -741,11 +859,12 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_packed_ker
 
 template <int BM, int BN>
 constexpr size_t packed_smem_bytes() {
-  return sizeof(float2) * 2 * BK * BM + sizeof(float) * 2 * BK * BN + sizeof(unsigned) * 6;
+  return sizeof(float2) * 2 * BK * BM + sizeof(float) * 2 * BK * BN + sizeof(unsigned) * 8;
 }
 
 // Launch entry of one (quantiser mode, order mode) family; defined once per translation unit.
-// tile: 0 = 128x128 (8x8), 1 = 128x64 (8x4), 2 = 64x64 (4x4), 3 = 32x32 (4x4... see table)
+// tile: 0 = 128x128 (8x8 per thread), 1 = 128x64 (8x4), 2 = 64x64 (4x4), 3 = 32x32 (4x4, 64 threads).
+// (The 8x8 micro-tile in CTAs of 64 or 128 threads was measured too: slower than 1..3 on every shape tried.)
 struct TileInfo { int bm, bn, tm, tn; };
 constexpr int TILE_COUNT = 4;
 __host__ inline TileInfo tile_info(int t) {
