@@ -172,6 +172,9 @@ struct RowLoader {
   bool row_ok[LPT];
   int ih0[LPT], iw0[LPT];               // conv: top-left input coordinate of the receptive field
   int ld_kh = 0, ld_kw = 0, ld_c0 = 0;  // conv vector path: position of the next slab inside (kh, kw, c_in)
+  // conv byte-wise path: for one output position and one kh, the taps (kw, c_in) are KW*C_in contiguous
+  // bytes of the input row ih0 + kh; the cursor is (kh, offset inside that run) of the next slab's first k
+  int any_kh = 0, any_off = 0;
 
   __device__ __forceinline__ void init(const Problem& p, int tid, int64_t m0, int64_t n0) {
 #pragma unroll
@@ -225,28 +228,52 @@ struct RowLoader {
             v = __ldg(reinterpret_cast<const uint4*>(row_ptr[l] + ((int64_t)ih * p.W + iw) * p.Cin + ld_c0));
         } else {  // LD_ANY: byte-wise, any K, any alignment, GEMM or conv
           uint32_t w4[4] = {0u, 0u, 0u, 0u};
+          if (!is_a || !p.is_conv) {
 #pragma unroll
-          for (int j = 0; j < BK; ++j) {
-            const int64_t k = k0 + j;
-            uint32_t byte = 0u;
-            if (k < K) {
-              if (!is_a || !p.is_conv) {
-                byte = __ldg(row_ptr[l] + k);
-              } else {
-                const int ci = (int)(k % p.Cin);
-                const int t = (int)(k / p.Cin);
-                const int kw = t % p.KW, kh = t / p.KW;
-                const int ih = ih0[l] + kh, iw = iw0[l] + kw;
-                if (ih >= 0 && ih < p.H && iw >= 0 && iw < p.W)
-                  byte = __ldg(row_ptr[l] + ((int64_t)ih * p.W + iw) * p.Cin + ci);
+            for (int j = 0; j < BK; ++j) {
+              const int64_t k = k0 + j;
+              const uint32_t byte = k < K ? (uint32_t)__ldg(row_ptr[l] + k) : 0u;
+              w4[j >> 2] |= byte << (8 * (j & 3));
+            }
+          } else {
+            // walk the runs: no division per byte.  Bytes of a run are valid where the tap column
+            // iw0 + kw lies inside the image, i.e. for run offsets in [lo, lo + span)
+            const int run = p.KW * p.Cin;
+            const int kw_lo = iw0[l] < 0 ? -iw0[l] : 0;
+            const int kw_hi = p.W - iw0[l] < p.KW ? p.W - iw0[l] : p.KW;
+            const int lo = kw_lo * p.Cin;
+            const unsigned span = kw_hi > kw_lo ? (unsigned)((kw_hi - kw_lo) * p.Cin) : 0u;
+            const int64_t row_pitch = (int64_t)p.W * p.Cin;
+            int off = any_off;
+            int ih = ih0[l] + any_kh;
+            // address of run offset 0 of input row ih (left of the image when iw0 < 0; only valid bytes are read)
+            int64_t pos = (int64_t)ih * row_pitch + (int64_t)iw0[l] * p.Cin + off;
+#pragma unroll
+            for (int j = 0; j < BK; ++j) {
+              const bool ok = (k0 + j < K) && ((unsigned)ih < (unsigned)p.H) && ((unsigned)(off - lo) < span);
+              const uint32_t byte = ok ? (uint32_t)__ldg(row_ptr[l] + pos) : 0u;
+              w4[j >> 2] |= byte << (8 * (j & 3));
+              ++off;
+              ++pos;
+              if (off == run) {
+                off = 0;
+                ++ih;
+                pos += row_pitch - run;
               }
             }
-            w4[j >> 2] |= byte << (8 * (j & 3));
           }
           v = make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
       }
       raw[l] = v;
+    }
+    if (LD == LD_ANY && p.is_conv) {  // advance the run cursor by one slab
+      const int run = p.KW * p.Cin;
+      any_off += BK;
+      while (any_off >= run) {
+        any_off -= run;
+        ++any_kh;
+      }
     }
     if (LD == LD_CONV_VEC) {  // advance (kh, kw, c0) to the next slab
       ld_c0 += BK;
