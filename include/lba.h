@@ -156,7 +156,7 @@ int lba_gemm_host_static(const uint8_t* A, const uint8_t* B, const float* scale_
 int lba_count_nan_codes(const uint8_t* codes, int64_t n, unsigned long long* count, void* stream);
 
 /* Which kernel variant a call with these arguments would run, as text, e.g.
- * "tile=128x128x16 micro=8x8 q=floor_fast order=chunk_slab load=gemm_vec grid=64x64".
+ * "tile=64x64x16 micro=4x8 q=floor_fast order=chunk16 load=gemm_vec grid=128x128".
  * is_conv selects the loader family; for a convolution pass M = B*H_out*W_out, N = C_out,
  * K = KH*KW*C_in and vec_ok = (C_in % 16 == 0 and pointers aligned).  Returns LBA_OK or the
  * error the real call would return; buf may be NULL. */

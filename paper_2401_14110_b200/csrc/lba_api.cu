@@ -187,14 +187,16 @@ bool packed_plan(int qm, int ord) { return qm == QM_FLOOR_FAST && ord != ORD_CHU
 
 int choose_tile(int64_t M, int64_t N, int qm, int ord) {
   (void)qm;
-  (void)ord;
   if (g_tile_override >= 0) return g_tile_override;
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) {
     int v = 0;
     if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
   }
-  const double eff[TILE_COUNT] = {1.00, 0.96, 0.88, 0.87};
+  // relative MAC rate of each tile with every SM loaded (8192^2 x 1024 and 4096 x 3072 x 768 GEMMs)
+  const double eff_seq[TILE_COUNT] = {1.00, 0.91, 0.95, 0.84};
+  const double eff_chunk[TILE_COUNT] = {0.97, 0.96, 1.00, 0.89};
+  const double* eff = ord == ORD_SEQ ? eff_seq : eff_chunk;
   int best = 0;
   double best_cost = 1e300;
   for (int t = 0; t < TILE_COUNT; ++t) {

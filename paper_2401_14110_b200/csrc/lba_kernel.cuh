@@ -890,12 +890,14 @@ constexpr size_t packed_smem_bytes() {
 }
 
 // Launch entry of one (quantiser mode, order mode) family; defined once per translation unit.
-// tile: 0 = 128x128 (8x8 per thread), 1 = 128x64 (8x4), 2 = 64x64 (4x4), 3 = 32x32 (4x4, 64 threads).
-// (The 8x8 micro-tile in CTAs of 64 or 128 threads was measured too: slower than 1..3 on every shape tried.)
+// tile: 0 = 128x128 (8x8 per thread, 256 threads), 1 = 128x64 (4x8, 256 threads), 2 = 64x64 (4x8, 128 threads),
+// 3 = 32x32 (4x4, 64 threads).  Micro-tiles are wider than tall because only the A operand is stored twice:
+// a 4x8 micro-tile needs 2 + 2 shared loads per k-step, an 8x4 one 4 + 1.  Measured and dropped: 8x8 in CTAs of
+// 64 or 128 threads, 4x8 in 32x64, 32x128, 64x128, 128x128, 64x256 tiles, a one-warp 32x32 tile.
 struct TileInfo { int bm, bn, tm, tn; };
 constexpr int TILE_COUNT = 4;
 __host__ inline TileInfo tile_info(int t) {
-  const TileInfo tab[TILE_COUNT] = {{128, 128, 8, 8}, {128, 64, 8, 4}, {64, 64, 4, 4}, {32, 32, 4, 4}};
+  const TileInfo tab[TILE_COUNT] = {{128, 128, 8, 8}, {128, 64, 4, 8}, {64, 64, 4, 8}, {32, 32, 4, 4}};
   return tab[t];
 }
 
