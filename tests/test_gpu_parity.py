@@ -129,6 +129,31 @@ def test_saturation_and_underflow_are_exercised():
     assert_bit_equal(got, ref_gemm(Amix, Bpos, one, one, None, prod, acc, CHK, 16))
 
 
+@pytest.mark.parametrize("tile", [0, 2, 3])
+def test_slow_climb_to_saturation_crosses_every_clamp_decision(tile):
+    # small same-sign products: each chunk adds a little, so the second-level sum creeps up to R_OF over many
+    # chunks.  On the way the kernel's running bound first skips the clamp, then measures the sums, then clamps
+    # for good; the sequential order does the same with its first-level bound.  All of it must stay exact.
+    prod, acc = code_domain_formats(7, 4)
+    M, N, K = 96, 80, 4096
+    a = (synth.gaussian((M, K), 81).abs() * 0.25 + 0.05) * torch.linspace(0.2, 1.2, M)[:, None]
+    b = synth.gaussian((N, K), 82).abs() * 0.25 + 0.05
+    a[:, ::97] *= -1.0                                   # a few negative taps so sums also step back
+    A = synth.e4m3_encode(a * 448.0 / 4.0)
+    B = synth.e4m3_encode(b * 448.0 / 4.0)
+    one = torch.ones(1)
+    lba.set_tile_override(tile)
+    try:
+        for order, chunk in ((CHK, 16), (SEQ, 16), (CHK, 64)):
+            got = gpu_gemm(A, B, one, one, None, prod, acc, order, chunk).cpu().numpy()
+            assert_bit_equal(got, ref_gemm(A, B, one, one, None, prod, acc, order, chunk), f"tile {tile} {order}/{chunk}")
+            if order == CHK and chunk == 16:
+                frac = float((got == np.float32(acc.r_of)).mean())
+                assert 0.02 < frac < 0.98, frac          # some outputs saturate, some do not
+    finally:
+        lba.set_tile_override(-1)
+
+
 def test_zero_and_empty_shapes():
     prod, acc = code_domain_formats(7, 4)
     one = torch.ones(1)
