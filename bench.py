@@ -316,13 +316,10 @@ def main():
     stop.record()
     barrier()
     clocks = sampler.stop()
-    total_ms = start.elapsed_time(stop)
-    if dist is not None:
-        t = torch.tensor([total_ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    from paper_2401_14110_b200 import sharding
+    total_ms = sharding.max_over_ranks(start.elapsed_time(stop), dist, device)
     ms_per_step = total_ms / args.steps
-    value = world * step_macs / (ms_per_step * 1e-3) / 1e9
+    value = sharding.whole_job_rate(step_macs, world, ms_per_step * 1e-3) / 1e9
 
     # ---- per-kernel accounting from the per-launch events
     per_call_ms = [statistics.mean(events[s][i][0].elapsed_time(events[s][i][1]) for s in range(args.steps))
@@ -397,11 +394,8 @@ def main():
             e2e_step()
         barrier()
         e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e = {"value": world * step_macs / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e_ms = sharding.max_over_ranks(e2e_ms, dist, device)
+        e2e = {"value": sharding.whole_job_rate(step_macs, world, e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
                "api": "lba_conv2d_host / lba_gemm_host (pinned host buffers, caller-owned device workspaces, "
                       "3 streams round-robin)"}
