@@ -14,7 +14,7 @@ namespace lba {
 // one definition per (QM, ORD), in the lba_fam_*.cu translation units
 #define LBA_DECL(QM, ORD) template <> cudaError_t launch_family<QM, ORD>(int, int, const Problem&, cudaStream_t);
 LBA_DECL(QM_FLOOR_FAST, ORD_SEQ) LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK_SLAB) LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK_ANY)
-LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK16)
+LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK16) LBA_DECL(QM_FLOOR_FULL, ORD_CHUNK16)
 LBA_DECL(QM_FLOOR_FULL, ORD_SEQ) LBA_DECL(QM_FLOOR_FULL, ORD_CHUNK_SLAB) LBA_DECL(QM_FLOOR_FULL, ORD_CHUNK_ANY)
 LBA_DECL(QM_RNE_FULL, ORD_SEQ) LBA_DECL(QM_RNE_FULL, ORD_CHUNK_SLAB) LBA_DECL(QM_RNE_FULL, ORD_CHUNK_ANY)
 LBA_DECL(QM_RNE_WIDE, ORD_SEQ) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_SLAB) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_ANY)
@@ -31,12 +31,12 @@ int cuda_fail(cudaError_t e) {
 }
 
 const LaunchFn kLaunch[QM_COUNT][ORD_COUNT] = {
-    // last column: chunk == 16 has a kernel of its own only for the fast floor quantiser (the plan never
+    // last column: chunk == 16 has a kernel of its own only for the floor quantisers (the plan never
     // selects it for the others; their entries repeat the general chunk-of-slabs family)
     {launch_family<QM_FLOOR_FAST, ORD_SEQ>, launch_family<QM_FLOOR_FAST, ORD_CHUNK_SLAB>,
      launch_family<QM_FLOOR_FAST, ORD_CHUNK_ANY>, launch_family<QM_FLOOR_FAST, ORD_CHUNK16>},
     {launch_family<QM_FLOOR_FULL, ORD_SEQ>, launch_family<QM_FLOOR_FULL, ORD_CHUNK_SLAB>,
-     launch_family<QM_FLOOR_FULL, ORD_CHUNK_ANY>, launch_family<QM_FLOOR_FULL, ORD_CHUNK_SLAB>},
+     launch_family<QM_FLOOR_FULL, ORD_CHUNK_ANY>, launch_family<QM_FLOOR_FULL, ORD_CHUNK16>},
     {launch_family<QM_RNE_FULL, ORD_SEQ>, launch_family<QM_RNE_FULL, ORD_CHUNK_SLAB>,
      launch_family<QM_RNE_FULL, ORD_CHUNK_ANY>, launch_family<QM_RNE_FULL, ORD_CHUNK_SLAB>},
     {launch_family<QM_RNE_WIDE, ORD_SEQ>, launch_family<QM_RNE_WIDE, ORD_CHUNK_SLAB>,
@@ -172,7 +172,7 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
   if (order == LBA_ORDER_SEQUENTIAL || (int64_t)chunk >= K) {
     pl->ord = ORD_SEQ;  // a single chunk: the second hierarchy adds it to 0, which changes nothing
   } else if (chunk % BK == 0) {
-    pl->ord = (chunk == BK && pl->qm == QM_FLOOR_FAST) ? ORD_CHUNK16 : ORD_CHUNK_SLAB;
+    pl->ord = (chunk == BK && (pl->qm == QM_FLOOR_FAST || pl->qm == QM_FLOOR_FULL)) ? ORD_CHUNK16 : ORD_CHUNK_SLAB;
     pl->chunk_slabs = chunk / BK;
   } else {
     pl->ord = ORD_CHUNK_ANY;
@@ -183,8 +183,6 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
 // Tile choice.  All CTAs of a launch have the same work and K is never split, so the launch ends when the
 // busiest SM has run its ceil(CTAs / SMs) tiles; larger tiles spend fewer instructions per MAC (eff, measured
 // on B200 with every SM loaded), smaller ones fill the SMs more evenly.  Pick the cheapest by that model.
-bool packed_plan(int qm, int ord) { return qm == QM_FLOOR_FAST && ord != ORD_CHUNK_ANY; }
-
 int choose_tile(int64_t M, int64_t N, int qm, int ord) {
   (void)qm;
   if (g_tile_override >= 0) return g_tile_override;

@@ -540,7 +540,11 @@ __host__ __device__ constexpr int packed_tmem_cols() {
 
 // the 8x8 micro-tile is held to 128 registers (two CTAs of 256 threads per SM) wherever the second-level
 // sums are not in registers
-template <int BM, int BN, int TM, int TN, int ORD, int LD>
+// PQ: what Q_prod has to do beyond the flush (the host proves which cases are reachable): nothing, cut the
+// mantissa (M_prod < 7), or cut and saturate (448^2 >= R_OF_prod)
+enum PackedProd { PQ_NONE = 0, PQ_MASK = 1, PQ_MASK_SAT = 2 };
+
+template <int BM, int BN, int TM, int TN, int PQ, int ORD, int LD>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN), (TM * TN == 64 && ORD != ORD_CHUNK_SLAB) ? 512 / ((BM / TM) * (BN / TN)) : 1)
     lba_contract_packed_kernel(const Problem p) {
   constexpr int NT = (BM / TM) * (BN / TN);
@@ -624,6 +628,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), (TM * TN == 64 && ORD !
   const u64 cc2 = pack2(p.c, p.c);
   const uint32_t mask = p.qa.mask;
   const float sat = p.qa.sat;
+  const uint32_t pmask = p.qp.mask;
+  const float psat = p.qp.sat;
 
   // one slab of 16 k-steps; CLAMP selects whether the magnitude clamp of Eq. 2 is applied.  The clamped
   // variant is the rare one and stays a rolled loop.  In chunk-16 order the slab starts a chunk: its first
@@ -649,7 +655,18 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), (TM * TN == 64 && ORD !
       for (int i = 0; i < TM; ++i)
 #pragma unroll
         for (int j = 0; j < PN; ++j) {
-          const u64 pr = mul2_ftz(a2[i], b2[j]);
+          u64 pr = mul2_ftz(a2[i], b2[j]);
+          if (PQ != PQ_NONE) {  // floor of Eq. 2 on the exact product, then its saturation
+            float plo, phi;
+            unpack2(pr, plo, phi);
+            plo = and_bits(plo, pmask);
+            phi = and_bits(phi, pmask);
+            if (PQ == PQ_MASK_SAT) {
+              plo = clamp_mag(plo, psat);
+              phi = clamp_mag(phi, psat);
+            }
+            pr = pack2(plo, phi);
+          }
           const u64 t = (CH16 && kk == 0) ? mul2_rz_ftz(pr, cc2) : fma2_rz_ftz(pr, cc2, acc1[i][j]);
           float lo, hi;
           unpack2(t, lo, hi);
