@@ -14,7 +14,7 @@ namespace lba {
 // one definition per (QM, ORD), in the lba_fam_*.cu translation units
 #define LBA_DECL(QM, ORD) template <> cudaError_t launch_family<QM, ORD>(int, int, const Problem&, cudaStream_t);
 LBA_DECL(QM_FLOOR_FAST, ORD_SEQ) LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK_SLAB) LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK_ANY)
-LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK16) LBA_DECL(QM_FLOOR_FULL, ORD_CHUNK16)
+LBA_DECL(QM_FLOOR_FAST, ORD_CHUNK16) LBA_DECL(QM_FLOOR_FULL, ORD_CHUNK16) LBA_DECL(QM_RNE_FULL, ORD_CHUNK16)
 LBA_DECL(QM_FLOOR_FULL, ORD_SEQ) LBA_DECL(QM_FLOOR_FULL, ORD_CHUNK_SLAB) LBA_DECL(QM_FLOOR_FULL, ORD_CHUNK_ANY)
 LBA_DECL(QM_RNE_FULL, ORD_SEQ) LBA_DECL(QM_RNE_FULL, ORD_CHUNK_SLAB) LBA_DECL(QM_RNE_FULL, ORD_CHUNK_ANY)
 LBA_DECL(QM_RNE_WIDE, ORD_SEQ) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_SLAB) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_ANY)
@@ -38,7 +38,7 @@ const LaunchFn kLaunch[QM_COUNT][ORD_COUNT] = {
     {launch_family<QM_FLOOR_FULL, ORD_SEQ>, launch_family<QM_FLOOR_FULL, ORD_CHUNK_SLAB>,
      launch_family<QM_FLOOR_FULL, ORD_CHUNK_ANY>, launch_family<QM_FLOOR_FULL, ORD_CHUNK16>},
     {launch_family<QM_RNE_FULL, ORD_SEQ>, launch_family<QM_RNE_FULL, ORD_CHUNK_SLAB>,
-     launch_family<QM_RNE_FULL, ORD_CHUNK_ANY>, launch_family<QM_RNE_FULL, ORD_CHUNK_SLAB>},
+     launch_family<QM_RNE_FULL, ORD_CHUNK_ANY>, launch_family<QM_RNE_FULL, ORD_CHUNK16>},
     {launch_family<QM_RNE_WIDE, ORD_SEQ>, launch_family<QM_RNE_WIDE, ORD_CHUNK_SLAB>,
      launch_family<QM_RNE_WIDE, ORD_CHUNK_ANY>, launch_family<QM_RNE_WIDE, ORD_CHUNK_SLAB>},
 };
@@ -55,6 +55,8 @@ struct Plan {
   int qm, ord;
   float dec_a, dec_b, c, un1, un2;
   float pk_a, pk_b, nrm_scale, inv_top;
+  int pq, rne_packed;
+  float rne_k_acc, rne_k_prod;
   QConst qp, qa;
   int chunk_slabs, chunk;
 };
@@ -166,13 +168,27 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
     }
   }
 
+  // ---- packed kernel: what Q_prod does beyond the flush; nearest-even rounds on the FP32 pipe by adding
+  // 1.5 * 2^(23-M) * 2^e, which needs that much exponent headroom above the largest carried magnitude
+  pl->pq = p_sat ? PQ_MASK_SAT : (p_round ? PQ_MASK : PQ_NONE);
+  pl->rne_k_acc = (float)std::ldexp(1.5, 23 - af->man_bits);
+  pl->rne_k_prod = (float)std::ldexp(1.5, 23 - pf->man_bits);
+  pl->rne_packed = 0;
+  if (pl->qm == QM_RNE_FULL) {
+    const int top_acc = (a_sat ? a_emax + 1 : (int)std::ceil(std::log2(max_sum)) + 1) + ka;
+    const int top_prod = 18 + kp;
+    pl->rne_packed = (top_acc + 25 - af->man_bits <= 127) && (top_prod + 25 - pf->man_bits <= 127) &&
+                     af->man_bits <= 21 && pf->man_bits <= 21;
+  }
+
   // ---- order mode
   pl->chunk = chunk;
   pl->chunk_slabs = 0;
   if (order == LBA_ORDER_SEQUENTIAL || (int64_t)chunk >= K) {
     pl->ord = ORD_SEQ;  // a single chunk: the second hierarchy adds it to 0, which changes nothing
   } else if (chunk % BK == 0) {
-    pl->ord = (chunk == BK && (pl->qm == QM_FLOOR_FAST || pl->qm == QM_FLOOR_FULL)) ? ORD_CHUNK16 : ORD_CHUNK_SLAB;
+    const bool packed = pl->qm == QM_FLOOR_FAST || pl->qm == QM_FLOOR_FULL || (pl->qm == QM_RNE_FULL && pl->rne_packed);
+    pl->ord = (chunk == BK && packed) ? ORD_CHUNK16 : ORD_CHUNK_SLAB;
     pl->chunk_slabs = chunk / BK;
   } else {
     pl->ord = ORD_CHUNK_ANY;
@@ -237,6 +253,10 @@ void apply_plan(Problem* p, const Plan& pl) {
   p->pk_b = pl.pk_b;
   p->nrm_scale = pl.nrm_scale;
   p->inv_top = pl.inv_top;
+  p->pq = pl.pq;
+  p->rne_packed = pl.rne_packed;
+  p->rne_k_acc = pl.rne_k_acc;
+  p->rne_k_prod = pl.rne_k_prod;
 }
 
 bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0; }

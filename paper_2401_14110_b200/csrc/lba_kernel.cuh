@@ -67,6 +67,9 @@ struct Problem {
   float pk_a, pk_b;    // 2^sx, 2^sw: decoded value -> product-carrier operand
   float nrm_scale;     // 2^-(e_max_acc + 1), or 0 when the accumulator cannot saturate
   float inv_top;       // accumulator carrier -> fraction of 2^(e_max_acc + 1)
+  int pq;              // PackedProd: what Q_prod does beyond the flush
+  int rne_packed;      // nearest-even: 1 if the packed kernel's exponent headroom suffices
+  float rne_k_acc, rne_k_prod;  // 1.5 * 2^(23 - M) for the accumulator and the product format
 };
 
 // ------------------------------------------------------------------ scalar building blocks
@@ -490,6 +493,65 @@ __device__ __forceinline__ u64 fma2_rz_ftz(u64 a, u64 b, u64 c) {
   asm("fma.rz.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
   return d;
 }
+__device__ __forceinline__ u64 fma2_rm(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rm.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 fma2_rp(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rp.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 fma2_rn(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 fma2_rn_ftz(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rn.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 mul2_rn(u64 a, u64 b) {  // IEEE
+  u64 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ u64 add2_rn(u64 a, u64 b) {
+  u64 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// Nearest-even cut of a pair of binary32 values to M mantissa bits on the FP32 pipe: adding
+// K = 1.5 * 2^(23-M) * 2^e (e the value's own exponent, same sign) moves the value into a binade whose unit in
+// the last place is the target grid step, so the addition itself rounds to nearest-even; K/ulp is even, so the
+// tie rule carries over; subtracting K is exact.  `v` may carry a sticky last bit (round-to-odd image of a
+// longer exact value), which keeps the result that of rounding the exact value once (needs M <= 21).
+// `kc` = {1.5 * 2^(23-M)} x 2, `neg1` = {-1} x 2.  FTZ picks whether a subnormal result is flushed.
+template <bool FTZ>
+__device__ __forceinline__ u64 rne2_fp(u64 v, u64 kc, u64 neg1) {
+  uint32_t lo, hi;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+  u64 e;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(e) : "r"(lo & 0xFF800000u), "r"(hi & 0xFF800000u));
+  const u64 k = mul2_rn(e, kc);
+  const u64 r = add2_rn(v, k);
+  return FTZ ? fma2_rn_ftz(k, neg1, r) : fma2_rn(k, neg1, r);
+}
+// round-to-odd image of the exact a*b+c: the toward-zero result with its last bit set when the sum is inexact
+// (the downward and upward results then differ, and they differ in the last bit).  tz carries the flush: a sum
+// below the smallest normal reads as (signed) zero, with at most the sticky bit on top.
+__device__ __forceinline__ u64 fma2_round_to_odd_ftz(u64 a, u64 b, u64 c) {
+  const u64 tz = fma2_rz_ftz(a, b, c), tm = fma2_rm(a, b, c), tp = fma2_rp(a, b, c);
+  uint32_t zl, zh, ml, mh, pl, ph;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(zl), "=r"(zh) : "l"(tz));
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(ml), "=r"(mh) : "l"(tm));
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(pl), "=r"(ph) : "l"(tp));
+  u64 d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(zl | ((ml ^ pl) & 1u)), "r"(zh | ((mh ^ ph) & 1u)));
+  return d;
+}
 __device__ __forceinline__ u64 mul2_rz_ftz(u64 a, u64 b) {
   u64 d;
   asm("mul.rz.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
@@ -531,11 +593,11 @@ __device__ __forceinline__ u64 pack2u(uint32_t lo, uint32_t hi) {
 }
 
 // columns of tensor memory a CTA of the packed kernel allocates (0: second-level sums stay in registers)
-template <int BM, int BN, int TM, int TN, int ORD>
+template <int BM, int BN, int TM, int TN, bool RNE, int ORD>
 __host__ __device__ constexpr int packed_tmem_cols() {
   constexpr int warps = (BM / TM) * (BN / TN) / 32;
   constexpr int cols = ((warps + 3) / 4) * TM * TN;
-  return (ORD == ORD_CHUNK16 && TM == 8) ? (cols < 32 ? 32 : cols) : 0;
+  return (ORD == ORD_CHUNK16 && TM == 8 && !RNE) ? (cols < 32 ? 32 : cols) : 0;
 }
 
 // the 8x8 micro-tile is held to 128 registers (two CTAs of 256 threads per SM) wherever the second-level
@@ -544,8 +606,11 @@ __host__ __device__ constexpr int packed_tmem_cols() {
 // mantissa (M_prod < 7), or cut and saturate (448^2 >= R_OF_prod)
 enum PackedProd { PQ_NONE = 0, PQ_MASK = 1, PQ_MASK_SAT = 2 };
 
-template <int BM, int BN, int TM, int TN, int PQ, int ORD, int LD>
-__global__ void __launch_bounds__((BM / TM) * (BN / TN), (TM * TN == 64 && ORD != ORD_CHUNK_SLAB) ? 512 / ((BM / TM) * (BN / TN)) : 1)
+// RNE: nearest-even instead of floor (then PQ_MASK means "round the product to M_prod bits").  Nearest-even
+// can raise a magnitude, so the slab-level proof that the clamp is idle is not used: it always clamps.
+template <int BM, int BN, int TM, int TN, int PQ, bool RNE, int ORD, int LD>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN),
+                                  (TM * TN == 64 && ORD != ORD_CHUNK_SLAB && !RNE) ? 512 / ((BM / TM) * (BN / TN)) : 1)
     lba_contract_packed_kernel(const Problem p) {
   constexpr int NT = (BM / TM) * (BN / TN);
   constexpr int TX = BN / TN;
@@ -554,7 +619,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), (TM * TN == 64 && ORD !
   constexpr int PN = TN / 2;  // register pairs per micro-tile row
   constexpr bool CH16 = ORD == ORD_CHUNK16;  // every slab is exactly one chunk
   constexpr bool CHUNKED = ORD == ORD_CHUNK_SLAB || CH16;
-  constexpr int TMEM_COLS = packed_tmem_cols<BM, BN, TM, TN, ORD>();
+  constexpr int TMEM_COLS = packed_tmem_cols<BM, BN, TM, TN, RNE, ORD>();
   constexpr bool T_IN_TMEM = TMEM_COLS > 0;   // second-level sums in tensor memory
   constexpr bool T_IN_REGS = CHUNKED && !T_IN_TMEM;
   static_assert(!T_IN_TMEM || (TM * TN) % 16 == 0, "tensor-memory groups of 16 columns");
@@ -606,8 +671,10 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), (TM * TN == 64 && ORD !
             else Bs[buf][q * 4 + j][r - BM] = s;
           }
         }
-        const unsigned m = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(n2 * p.nrm_scale));
-        if ((tid & 31) == 0) atomicMax(&nrm[cell][is_a ? 0 : 1], m);
+        if (!RNE) {
+          const unsigned m = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(n2 * p.nrm_scale));
+          if ((tid & 31) == 0) atomicMax(&nrm[cell][is_a ? 0 : 1], m);
+        }
       }
     }
   };
@@ -630,13 +697,15 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), (TM * TN == 64 && ORD !
   const float sat = p.qa.sat;
   const uint32_t pmask = p.qp.mask;
   const float psat = p.qp.sat;
+  const u64 kc_acc = pack2(p.rne_k_acc, p.rne_k_acc), kc_prod = pack2(p.rne_k_prod, p.rne_k_prod);
+  const u64 neg1 = pack2(-1.0f, -1.0f);
 
   // one slab of 16 k-steps; CLAMP selects whether the magnitude clamp of Eq. 2 is applied.  The clamped
   // variant is the rare one and stays a rolled loop.  In chunk-16 order the slab starts a chunk: its first
   // step adds to zero, which is a plain (exact) scaling of the product, so the sums need no clearing.
   auto slab_body = [&](int buf, auto clamp_tag) {
     constexpr bool CLAMP = decltype(clamp_tag)::value;
-    constexpr int UNR = CLAMP ? 1 : KUNROLL;
+    constexpr int UNR = (CLAMP && !RNE) ? 1 : KUNROLL;
 #pragma unroll UNR
     for (int kk = 0; kk < BK; ++kk) {
       u64 a2[TM], b2[PN];
@@ -656,6 +725,21 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), (TM * TN == 64 && ORD !
 #pragma unroll
         for (int j = 0; j < PN; ++j) {
           u64 pr = mul2_ftz(a2[i], b2[j]);
+          if (RNE) {
+            if (PQ != PQ_NONE) {  // nearest-even on the exact product, then its saturation
+              pr = rne2_fp<false>(pr, kc_prod, neg1);
+              if (PQ == PQ_MASK_SAT) {
+                float plo, phi;
+                unpack2(pr, plo, phi);
+                pr = pack2(clamp_mag(plo, psat), clamp_mag(phi, psat));
+              }
+            }
+            const u64 ro = fma2_round_to_odd_ftz(pr, cc2, (CH16 && kk == 0) ? 0ull : acc1[i][j]);
+            float lo, hi;
+            unpack2(rne2_fp<true>(ro, kc_acc, neg1), lo, hi);
+            acc1[i][j] = pack2(clamp_mag(lo, sat), clamp_mag(hi, sat));
+            continue;
+          }
           if (PQ != PQ_NONE) {  // floor of Eq. 2 on the exact product, then its saturation
             float plo, phi;
             unpack2(pr, plo, phi);
@@ -691,9 +775,14 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), (TM * TN == 64 && ORD !
       for (int j = 0; j < PN; ++j) {
         u64& t2 = acc2[T_IN_REGS ? i : 0][T_IN_REGS ? j : 0];
         float lo, hi;
-        unpack2(add2_rz_ftz(acc1[i][j], t2), lo, hi);
-        lo = and_bits(lo, mask);
-        hi = and_bits(hi, mask);
+        if (RNE) {
+          const u64 one2 = pack2(1.0f, 1.0f);
+          unpack2(rne2_fp<true>(fma2_round_to_odd_ftz(acc1[i][j], one2, t2), kc_acc, neg1), lo, hi);
+        } else {
+          unpack2(add2_rz_ftz(acc1[i][j], t2), lo, hi);
+          lo = and_bits(lo, mask);
+          hi = and_bits(hi, mask);
+        }
         if (CLAMP) {
           lo = clamp_mag(lo, sat);
           hi = clamp_mag(hi, sat);
@@ -797,7 +886,17 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), (TM * TN == 64 && ORD !
     if (tid < 2) nrm[cell_clear][tid] = 0u;  // read during the previous slab, filled during the next
     // ||x|| ||w|| / 2^(e_max+1), rounded up generously (the norms carry rounding errors near 2^-20)
     const float grow = sqrtf(na * nb) * 1.01f;
-    if (CH16) {
+    if (RNE) {
+      slab_body(buf, std::true_type());
+      if (CH16) {
+        close_chunk(std::true_type());
+      } else if (CHUNKED) {
+        if (++slabs_in_chunk == p.chunk_slabs) {
+          close_chunk(std::true_type());
+          slabs_in_chunk = 0;
+        }
+      }
+    } else if (CH16) {
       // the chunk starts from zero, so the CTA-wide bound alone decides (same value in every thread)
       if (grow < 0.999f) slab_body(buf, std::false_type());
       else slab_body(buf, std::true_type());
