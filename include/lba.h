@@ -88,6 +88,18 @@ int lba_gemm(const uint8_t* A, const uint8_t* B, const float* scale_a, int scale
              int scale_b_len, const float* bias, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt,
              const lba_fmt* acc_fmt, int order, int chunk, float* out, void* stream);
 
+/* Batched GEMM: `batch` independent problems of the same shape and formats in one launch, problem z reading
+ * A + z*stride_a and B + z*stride_b (byte offsets; [M][K] and [N][K] each) and writing out + z*stride_out
+ * (offset in floats; [M][N]).  This is the matrix product inside attention (Q K^T and P V), which the paper
+ * also routes through the LBA GEMM (App. C.2: all fully connected layers and matrix multiplications).
+ * A stride of 0 shares that operand between all problems; otherwise strides must be at least one problem's
+ * size, and stride_out always.  Scales and bias are shared by all problems (same lengths as lba_gemm).
+ * Strides that are multiples of 16 keep the vector-load path. */
+int lba_gemm_batched(const uint8_t* A, const uint8_t* B, const float* scale_a, int scale_a_len, const float* scale_b,
+                     int scale_b_len, const float* bias, int64_t batch, int64_t M, int64_t N, int64_t K,
+                     int64_t stride_a, int64_t stride_b, int64_t stride_out, const lba_fmt* prod_fmt,
+                     const lba_fmt* acc_fmt, int order, int chunk, float* out, void* stream);
+
 /* Convolution as an implicit GEMM (Eq. 3 with m = (b, oh, ow), n = c_out and k walking
  * (kh, kw, c_in), c_in fastest).  Padded taps are the value 0 and still count toward the
  * chunk position.  Dilation 1, groups 1.

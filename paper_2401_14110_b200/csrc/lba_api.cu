@@ -199,7 +199,7 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
 // Tile choice.  All CTAs of a launch have the same work and K is never split, so the launch ends when the
 // busiest SM has run its ceil(CTAs / SMs) tiles; larger tiles spend fewer instructions per MAC (eff, measured
 // on B200 with every SM loaded), smaller ones fill the SMs more evenly.  Pick the cheapest by that model.
-int choose_tile(int64_t M, int64_t N, int qm, int ord) {
+int choose_tile(int64_t M, int64_t N, int64_t batch, int qm, int ord) {
   (void)qm;
   if (g_tile_override >= 0) return g_tile_override;
   int dev = 0, sms = 148;
@@ -215,7 +215,7 @@ int choose_tile(int64_t M, int64_t N, int qm, int ord) {
   double best_cost = 1e300;
   for (int t = 0; t < TILE_COUNT; ++t) {
     const TileInfo ti = tile_info(t);
-    const double ctas = (double)((M + ti.bm - 1) / ti.bm) * (double)((N + ti.bn - 1) / ti.bn);
+    const double ctas = (double)((M + ti.bm - 1) / ti.bm) * (double)((N + ti.bn - 1) / ti.bn) * (double)batch;
     const double per_sm = std::ceil(ctas / sms);
     double cost = per_sm * ti.bm * ti.bn / eff[t];
     if (t == 0 && per_sm < 2) cost /= 0.85;  // one 8-warp CTA alone does not keep an SM's pipes busy
@@ -262,8 +262,9 @@ void apply_plan(Problem* p, const Plan& pl) {
 bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0; }
 
 int run(const Problem& p, const Plan& pl, int load, cudaStream_t stream) {
-  if (p.M == 0 || p.N == 0) return LBA_OK;
-  const int tile = choose_tile(p.M, p.N, pl.qm, pl.ord);
+  if (p.M == 0 || p.N == 0 || p.batch == 0) return LBA_OK;
+  if (p.batch > 65535) return LBA_ERR_SHAPE;
+  const int tile = choose_tile(p.M, p.N, p.batch, pl.qm, pl.ord);
   const TileInfo ti = tile_info(tile);
   if ((p.N + ti.bn - 1) / ti.bn > 65535 || (p.M + ti.bm - 1) / ti.bm > 2147483647LL) return LBA_ERR_SHAPE;
   const cudaError_t e = kLaunch[pl.qm][pl.ord](tile, load, p, stream);
@@ -342,6 +343,7 @@ int lba_gemm(const uint8_t* A, const uint8_t* B, const float* scale_a, int scale
   p.M = M;
   p.N = N;
   p.K = K;
+  p.batch = 1;
   if ((st = fill_scales(&p, scale_a, scale_a_len, scale_b, scale_b_len, bias)) != LBA_OK) return st;
   if (M > 0 && N > 0 && !out) return LBA_ERR_NULL;
   if (K > 0 && ((M > 0 && !A) || (N > 0 && !B))) return LBA_ERR_NULL;
@@ -351,6 +353,46 @@ int lba_gemm(const uint8_t* A, const uint8_t* B, const float* scale_a, int scale
   apply_plan(&p, pl);
   const bool vec = K % BK == 0 && aligned16(A) && aligned16(B);
   return run(p, pl, vec ? LD_GEMM_VEC : LD_ANY, (cudaStream_t)stream);
+}
+
+int lba_gemm_batched(const uint8_t* A, const uint8_t* B, const float* scale_a, int scale_a_len, const float* scale_b,
+                     int scale_b_len, const float* bias, int64_t batch, int64_t M, int64_t N, int64_t K,
+                     int64_t stride_a, int64_t stride_b, int64_t stride_out, const lba_fmt* prod_fmt,
+                     const lba_fmt* acc_fmt, int order, int chunk, float* out, void* stream) {
+  if (batch < 0 || M < 0 || N < 0 || K < 0 || K > 2147483647LL) return LBA_ERR_SHAPE;
+  // problems may share an operand (stride 0) but outputs must not overlap
+  if (stride_a < 0 || stride_b < 0 || stride_out < 0) return LBA_ERR_SHAPE;
+  if (batch > 1 && ((stride_a != 0 && stride_a < M * K) || (stride_b != 0 && stride_b < N * K) || stride_out < M * N))
+    return LBA_ERR_SHAPE;
+  Plan pl;
+  int st = make_plan(prod_fmt, acc_fmt, order, chunk, K, &pl);
+  if (st != LBA_OK) return st;
+  Problem p;
+  std::memset(&p, 0, sizeof(p));
+  p.M = M;
+  p.N = N;
+  p.K = K;
+  if ((st = fill_scales(&p, scale_a, scale_a_len, scale_b, scale_b_len, bias)) != LBA_OK) return st;
+  if (batch > 0 && M > 0 && N > 0 && !out) return LBA_ERR_NULL;
+  if (batch > 0 && K > 0 && ((M > 0 && !A) || (N > 0 && !B))) return LBA_ERR_NULL;
+  p.A = A;
+  p.B = B;
+  p.out = out;
+  p.batch_a = stride_a;
+  p.batch_b = stride_b;
+  p.batch_out = stride_out;
+  apply_plan(&p, pl);
+  const bool vec = K % BK == 0 && aligned16(A) && aligned16(B) && stride_a % 16 == 0 && stride_b % 16 == 0;
+  // the grid's third dimension holds at most 65535 problems
+  for (int64_t b0 = 0; b0 < batch; b0 += 65535) {
+    Problem q = p;
+    q.batch = batch - b0 < 65535 ? batch - b0 : 65535;
+    q.A = A + b0 * stride_a;
+    q.B = B + b0 * stride_b;
+    q.out = out + b0 * stride_out;
+    if ((st = run(q, pl, vec ? LD_GEMM_VEC : LD_ANY, (cudaStream_t)stream)) != LBA_OK) return st;
+  }
+  return LBA_OK;
 }
 
 int lba_conv2d(const uint8_t* x, const uint8_t* w, const float* scale_x, int scale_x_len, const float* scale_w,
@@ -368,6 +410,7 @@ int lba_conv2d(const uint8_t* x, const uint8_t* w, const float* scale_x, int sca
   p.M = g.M;
   p.N = C_out;
   p.K = g.K;
+  p.batch = 1;
   if ((st = fill_scales(&p, scale_x, scale_x_len, scale_w, scale_w_len, bias)) != LBA_OK) return st;
   p.A = x;
   p.B = w;
@@ -494,7 +537,7 @@ int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, 
   Plan pl;
   const int st = make_plan(prod_fmt, acc_fmt, order, chunk, K, &pl);
   if (st != LBA_OK) return st;
-  const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, pl.qm, pl.ord);
+  const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, 1, pl.qm, pl.ord);
   const TileInfo ti = tile_info(tile);
   const int load = vec_ok ? (is_conv ? LD_CONV_VEC : LD_GEMM_VEC) : LD_ANY;
   if (buf && buf_len)

@@ -55,6 +55,9 @@ struct Problem {
   const float* bias;
   float* out;
   int64_t M, N, K;
+  // batched GEMM: problem z = blockIdx.z reads A + z*batch_a, B + z*batch_b (bytes) and writes out + z*batch_out
+  // (floats); a plain call has batch = 1
+  int64_t batch, batch_a, batch_b, batch_out;
   int sa_per_row, sb_per_col;
   int is_conv, H, W, Cin, KH, KW, sh, sw, ph, pw, Hout, Wout;
   float dec_a, dec_b;  // decode multipliers 2^(120+sx), 2^(120+sw)
@@ -180,6 +183,8 @@ struct RowLoader {
   int any_kh = 0, any_off = 0;
 
   __device__ __forceinline__ void init(const Problem& p, int tid, int64_t m0, int64_t n0) {
+    const uint8_t* const baseA = p.A + (int64_t)blockIdx.z * p.batch_a;
+    const uint8_t* const baseB = p.B + (int64_t)blockIdx.z * p.batch_b;
 #pragma unroll
     for (int l = 0; l < LPT; ++l) {
       const int r = tid + l * NT;
@@ -192,7 +197,7 @@ struct RowLoader {
         if (m < p.M) {
           row_ok[l] = true;
           if (LD == LD_GEMM_VEC || (LD == LD_ANY && !p.is_conv)) {
-            row_ptr[l] = p.A + m * p.K;
+            row_ptr[l] = baseA + m * p.K;
           } else {
             const int ow = (int)(m % p.Wout);
             const int64_t t = m / p.Wout;
@@ -200,14 +205,14 @@ struct RowLoader {
             const int64_t b = t / p.Hout;
             ih0[l] = oh * p.sh - p.ph;
             iw0[l] = ow * p.sw - p.pw;
-            row_ptr[l] = p.A + b * ((int64_t)p.H * p.W * p.Cin);
+            row_ptr[l] = baseA + b * ((int64_t)p.H * p.W * p.Cin);
           }
         }
       } else if (r < ROWS) {
         const int64_t n = n0 + (r - BM);
         if (n < p.N) {
           row_ok[l] = true;
-          row_ptr[l] = p.B + n * p.K;
+          row_ptr[l] = baseB + n * p.K;
         }
       }
     }
@@ -417,7 +422,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
   if (ORD == ORD_CHUNK_ANY && k_in_chunk > 0) close_chunk();
 
   // ---- epilogue: back to real values, +0 for every zero, scales and bias in binary32
-  const bool vec_store = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0);
+  float* const outz = p.out + (int64_t)blockIdx.z * p.batch_out;
+  const bool vec_store = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(outz) & 15) == 0);
 #pragma unroll
   for (int i = 0; i < TM; ++i) {
     const int64_t m = m0 + (i / 4) * (BM / 2) + ty * 4 + (i % 4);
@@ -444,7 +450,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
           if (p.bias) r = __fadd_rn(r, p.bias[n + j]);
           ov[j] = r;
         }
-        *reinterpret_cast<float4*>(p.out + m * p.N + n) = v;
+        *reinterpret_cast<float4*>(outz + m * p.N + n) = v;
       } else {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -452,7 +458,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
             const float sb = p.sb[p.sb_per_col ? n + j : 0];
             float r = __fmul_rn(__fmul_rn(o[j], sa), sb);
             if (p.bias) r = __fadd_rn(r, p.bias[n + j]);
-            p.out[m * p.N + n + j] = r;
+            outz[m * p.N + n + j] = r;
           }
         }
       }
@@ -954,7 +960,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
   }
 
   // ---- epilogue: back to real values, +0 for every zero, scales and bias in binary32
-  const bool vec_store = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0);
+  float* const outz = p.out + (int64_t)blockIdx.z * p.batch_out;
+  const bool vec_store = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(outz) & 15) == 0);
 #pragma unroll
   for (int i = 0; i < TM; ++i) {
     const int64_t m = m0 + (i / 4) * (BM / 2) + ty * 4 + (i % 4);
@@ -984,7 +991,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
           if (p.bias) r = __fadd_rn(r, p.bias[n + j]);
           ov[j] = r;
         }
-        *reinterpret_cast<float4*>(p.out + m * p.N + n) = v;
+        *reinterpret_cast<float4*>(outz + m * p.N + n) = v;
       } else {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -992,7 +999,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
             const float sb = p.sb[p.sb_per_col ? n + j : 0];
             float r = __fmul_rn(__fmul_rn(o[j], sa), sb);
             if (p.bias) r = __fadd_rn(r, p.bias[n + j]);
-            p.out[m * p.N + n + j] = r;
+            outz[m * p.N + n + j] = r;
           }
         }
       }

@@ -154,6 +154,52 @@ def test_slow_climb_to_saturation_crosses_every_clamp_decision(tile):
         lba.set_tile_override(-1)
 
 
+@pytest.mark.parametrize("case", [
+    (24, 128, 128, 64, False),     # attention scores Q K^T: 24 heads, 128 tokens, head size 64
+    (24, 128, 64, 128, False),     # attention output P V (V stored transposed)
+    (5, 70, 33, 37, False),        # nothing aligned: byte-wise loader, strides not multiples of 16
+    (7, 40, 96, 48, True),         # one B shared by every problem
+    (1, 50, 50, 16, False),
+])
+@pytest.mark.parametrize("name", ["m7e4_code", "m4e4_rne"])
+def test_batched_gemm_equals_one_gemm_per_problem(case, name):
+    Z, M, N, K, shared_b = case
+    prod, acc = FORMATS[name]
+    A = synth.e4m3_encode(synth.gaussian((Z, M, K), 91) * 100.0)
+    B = synth.e4m3_encode(synth.gaussian((N, K) if shared_b else (Z, N, K), 92) * 100.0)
+    sa = torch.tensor([0.01])
+    sb = torch.linspace(0.5, 1.5, N)
+    bias = torch.linspace(-1, 1, N)
+    for order, chunk in ((CHK, 16), (SEQ, 16)):
+        got = lba.lba_gemm_batched(A.to(DEV), B.to(DEV), sa.to(DEV), sb.to(DEV), bias.to(DEV), prod, acc, order,
+                                   chunk).cpu().numpy()
+        assert got.shape == (Z, M, N)
+        for z in range(Z):
+            Bz = B if shared_b else B[z]
+            want = ref_gemm(A[z], Bz, sa, sb, bias, prod, acc, order, chunk)
+            assert_bit_equal(got[z], want, f"{case} {name} problem {z} order {order}")
+
+
+def test_batched_gemm_argument_checks():
+    prod, acc = code_domain_formats(7, 4)
+    one = torch.ones(1, device=DEV)
+    A = synth.random_codes((3, 8, 16), 1).to(DEV)
+    B = synth.random_codes((3, 8, 16), 2).to(DEV)
+    assert lba.lba_gemm_batched(A[:0], B[:0], one, one, None, prod, acc).shape == (0, 8, 8)
+    lib = lba.load_library()
+    import ctypes as C
+    pf, af = lba._fmt(prod), lba._fmt(acc)
+    out = torch.empty((3, 8, 8), dtype=torch.float32, device=DEV)
+    args = lambda sa_, sb_, so_: (C.c_void_p(A.data_ptr()), C.c_void_p(B.data_ptr()), C.c_void_p(one.data_ptr()), 1,
+                                  C.c_void_p(one.data_ptr()), 1, None, 3, 8, 8, 16, sa_, sb_, so_, C.byref(pf),
+                                  C.byref(af), CHK, 16, C.c_void_p(out.data_ptr()), None)
+    assert lib.lba_gemm_batched(*args(128, 128, 64)) == 0
+    assert lib.lba_gemm_batched(*args(128, 128, 63)) == -2     # outputs would overlap
+    assert lib.lba_gemm_batched(*args(100, 128, 64)) == -2     # A problems would overlap
+    assert lib.lba_gemm_batched(*args(0, 0, 64)) == 0          # shared operands are fine
+    torch.cuda.synchronize()
+
+
 def test_zero_and_empty_shapes():
     prod, acc = code_domain_formats(7, 4)
     one = torch.ones(1)
