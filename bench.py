@@ -61,6 +61,9 @@ def parse_args():
                     help="size of the oracle sample timed for cpu_baseline (emulated MACs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--force-dist", action="store_true",
+                    help="initialise torch.distributed (NCCL) even for a single rank: exercises the multi-GPU plumbing "
+                         "(barrier, max over ranks) on one GPU")
     return ap.parse_args()
 
 
@@ -277,9 +280,11 @@ def main():
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     dist = None
-    if world > 1:
+    if world > 1 or args.force_dist:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=device)
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29511")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=device)
 
     from paper_2401_14110_b200 import binding as lba
     ORDER_CHUNKED = RUN_ORDER
