@@ -176,9 +176,15 @@ int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, 
                       int chunk, int is_conv, int vec_ok, char* buf, size_t buf_len);
 
 /* Testing and tuning hook: force the CTA tile (0 = 128x128, 1 = 128x64, 2 = 64x64, 3 = 32x32
- * outputs; -1 = automatic choice, the default).  Process-wide; results never depend on the tile,
+ * outputs; 4 = the experimental kernel whose products come from the tensor cores, 128x64 outputs, used only
+ * for the fast floor quantiser in chunk-16 order and ignored otherwise; -1 = automatic choice, the default).  Process-wide; results never depend on the tile,
  * only speed does.  Returns LBA_OK, or LBA_ERR_SHAPE for an unknown tile. */
 int lba_set_tile_override(int tile);
+
+/* Error word of the device code: kernels that wait on hardware barriers bound every wait, and a wait that runs
+ * out stores a non-zero code here instead of hanging.  Reads and clears the word; synchronises the device.
+ * 0 means no kernel has reported a problem since the last call. */
+int lba_device_error(int* code);
 
 const char* lba_status_string(int status);
 int lba_last_cuda_error(void); /* cudaError_t of the most recent failed CUDA call in this thread, else 0 */

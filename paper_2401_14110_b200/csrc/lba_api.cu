@@ -20,6 +20,9 @@ LBA_DECL(QM_RNE_FULL, ORD_SEQ) LBA_DECL(QM_RNE_FULL, ORD_CHUNK_SLAB) LBA_DECL(QM
 LBA_DECL(QM_RNE_WIDE, ORD_SEQ) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_SLAB) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_ANY)
 #undef LBA_DECL
 
+cudaError_t launch_umma_family(int load, const Problem& p, cudaStream_t stream);
+cudaError_t read_umma_error(int* code);
+
 namespace {
 
 thread_local int g_last_cuda_error = 0;
@@ -201,7 +204,7 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
 // on B200 with every SM loaded), smaller ones fill the SMs more evenly.  Pick the cheapest by that model.
 int choose_tile(int64_t M, int64_t N, int64_t batch, int qm, int ord) {
   (void)qm;
-  if (g_tile_override >= 0) return g_tile_override;
+  if (g_tile_override >= 0 && g_tile_override < TILE_COUNT) return g_tile_override;
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) {
     int v = 0;
@@ -264,6 +267,13 @@ bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15)
 int run(const Problem& p, const Plan& pl, int load, cudaStream_t stream) {
   if (p.M == 0 || p.N == 0 || p.batch == 0) return LBA_OK;
   if (p.batch > 65535) return LBA_ERR_SHAPE;
+  if (g_tile_override == TILE_UMMA) {  // the tensor-core-product kernel, where it applies
+    if (pl.qm == QM_FLOOR_FAST && pl.ord == ORD_CHUNK16) {
+      if ((p.N + 63) / 64 > 65535) return LBA_ERR_SHAPE;
+      const cudaError_t e = launch_umma_family(load, p, stream);
+      return e == cudaSuccess ? LBA_OK : cuda_fail(e);
+    }
+  }
   const int tile = choose_tile(p.M, p.N, p.batch, pl.qm, pl.ord);
   const TileInfo ti = tile_info(tile);
   if ((p.N + ti.bn - 1) / ti.bn > 65535 || (p.M + ti.bm - 1) / ti.bm > 2147483647LL) return LBA_ERR_SHAPE;
@@ -308,10 +318,16 @@ extern "C" {
 
 int lba_version(void) { return 1; }
 
+int lba_device_error(int* code) {
+  if (!code) return LBA_ERR_NULL;
+  const cudaError_t e = read_umma_error(code);
+  return e == cudaSuccess ? LBA_OK : cuda_fail(e);
+}
+
 int lba_last_cuda_error(void) { return g_last_cuda_error; }
 
 int lba_set_tile_override(int tile) {
-  if (tile < -1 || tile >= TILE_COUNT) return LBA_ERR_SHAPE;
+  if (tile < -1 || tile > TILE_UMMA) return LBA_ERR_SHAPE;
   g_tile_override = tile;
   return LBA_OK;
 }

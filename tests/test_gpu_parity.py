@@ -200,6 +200,27 @@ def test_batched_gemm_argument_checks():
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("shape", [(128, 64, 16), (200, 100, 37), (513, 130, 576), (1000, 64, 2304)])
+def test_tensor_core_product_kernel_is_exact(shape):
+    # tile override 4: the products come from tcgen05.mma (one non-zero k per MMA), the CUDA cores only add,
+    # mask and clamp.  Not chosen automatically (measured slower than the packed kernel); it must still be exact,
+    # and none of its bounded waits may run out.
+    M, N, K = shape
+    prod, acc = code_domain_formats(7, 4)
+    A, sa, B, sb = synth.gemm_case(M, N, K, config=95)
+    bias = torch.linspace(-1, 1, N)
+    assert lba.device_error() == 0
+    lba.set_tile_override(4)
+    try:
+        got = gpu_gemm(A, B, sa, sb, bias, prod, acc, CHK, 16)
+        pos = gpu_gemm(A & 0x7F, B & 0x7F, sa, sb, None, prod, acc, CHK, 16)     # saturating: the clamped variants
+    finally:
+        lba.set_tile_override(-1)
+    assert lba.device_error() == 0
+    assert_bit_equal(got, ref_gemm(A, B, sa, sb, bias, prod, acc, CHK, 16), f"umma {shape}")
+    assert_bit_equal(pos, ref_gemm(A & 0x7F, B & 0x7F, sa, sb, None, prod, acc, CHK, 16), f"umma saturating {shape}")
+
+
 def test_zero_and_empty_shapes():
     prod, acc = code_domain_formats(7, 4)
     one = torch.ones(1)
