@@ -55,8 +55,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet18",
-                    help="resnet18 (default, the benchmark) or gemm:MxNxK[:seq|chunk], one LBA GEMM on Gaussian "
-                         "operands (used for kernel profiles)")
+                    help="resnet18 (default, the benchmark), gemm:MxNxK[:seq|chunk] (one LBA GEMM on Gaussian "
+                         "operands, used for kernel profiles) or bgemm:ZxMxNxK[:seq|chunk] (one batched call)")
     ap.add_argument("--cpu-baseline-macs", type=float, default=1.5e9,
                     help="size of the oracle sample timed for cpu_baseline (emulated MACs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -138,6 +138,14 @@ def formats():
 def build_calls(device):
     from paper_2401_14110_b200 import binding as lba, synth, workloads, ORDER_CHUNKED
     prod, acc = formats()
+    if GEMM_CASE is not None and len(GEMM_CASE) == 4:      # batched: Z problems of M x N x K (attention matmuls)
+        z, m, n, k = GEMM_CASE
+        a = synth.e4m3_encode(synth.gaussian((z, m, k), synth.seed_for(5, 0)) * 100.0)
+        b = synth.e4m3_encode(synth.gaussian((z, n, k), synth.seed_for(5, 1)) * 100.0)
+        one = torch.ones(1, device=device)
+        c = workloads.LbaCall("bgemm", "bgemm", a.to(device), b.to(device), one, one)
+        c.out = torch.empty((z, m, n), dtype=torch.float32, device=device)
+        return [c]
     if GEMM_CASE is not None:
         m, n, k = GEMM_CASE
         a, sa, b, sb = synth.gemm_case(m, n, k, config=5)
@@ -167,6 +175,8 @@ def run_step(calls, events=None):
             events[i][0].record()
         if c.kind == "conv":
             lba.lba_conv2d(c.x, c.w, c.sx, c.sw, None, c.stride, c.pad, prod, acc, ORDER_CHUNKED, 16, out=c.out_nhwc)
+        elif c.kind == "bgemm":
+            lba.lba_gemm_batched(c.x, c.w, c.sx, c.sw, None, prod, acc, ORDER_CHUNKED, 16, out=c.out)
         else:
             lba.lba_gemm(c.x, c.w, c.sx, c.sw, None, prod, acc, ORDER_CHUNKED, 16, out=c.out)
         if events is not None:
@@ -262,7 +272,15 @@ def reference_arm(args):
 def main():
     global WORKLOAD, RUN_ORDER, GEMM_CASE
     args = parse_args()
-    if args.workload.startswith("gemm:"):
+    if args.workload.startswith("bgemm:"):
+        parts = args.workload.split(":")
+        GEMM_CASE = tuple(int(v) for v in parts[1].lower().split("x"))
+        if len(GEMM_CASE) != 4:
+            raise SystemExit("--workload bgemm:ZxMxNxK")
+        RUN_ORDER = 0 if (len(parts) > 2 and parts[2].startswith("seq")) else 1
+        WORKLOAD = "batched_lba_gemm_%dx%dx%dx%d_m7e4_%s" % (GEMM_CASE + ("sequential" if RUN_ORDER == 0 else "chunk16",))
+        args.no_e2e = args.no_cpu_baseline = True      # kernel timing only for this workload
+    elif args.workload.startswith("gemm:"):
         parts = args.workload.split(":")
         GEMM_CASE = tuple(int(v) for v in parts[1].lower().split("x"))
         RUN_ORDER = 0 if (len(parts) > 2 and parts[2].startswith("seq")) else 1

@@ -97,6 +97,8 @@ class LbaCall:
 
     @property
     def gemm_shape(self):
+        if self.kind == "bgemm":        # per problem; macs counts all of them
+            return self.x.shape[1], self.w.shape[1], self.x.shape[2]
         if self.kind == "gemm":
             return self.x.shape[0], self.w.shape[0], self.x.shape[1]
         b, h, wd, cin = self.x.shape
@@ -108,7 +110,7 @@ class LbaCall:
     @property
     def macs(self):
         m, n, k = self.gemm_shape
-        return m * n * k
+        return m * n * k * (self.x.shape[0] if self.kind == "bgemm" else 1)
 
 
 def _quant_act(t_nhwc: torch.Tensor):
