@@ -221,6 +221,52 @@ def test_tensor_core_product_kernel_is_exact(shape):
     assert_bit_equal(pos, ref_gemm(A & 0x7F, B & 0x7F, sa, sb, None, prod, acc, CHK, 16), f"umma saturating {shape}")
 
 
+def test_random_formats_shapes_orders_and_data_regimes():
+    # a seeded sweep over everything at once: shapes with ragged edges, mantissa / exponent / bias choices around
+    # the thresholds that switch kernel variants, floor and nearest-even, with and without the underflow branch,
+    # every order, chunk lengths that do and do not fit slabs, and input magnitudes from "everything underflows"
+    # to "everything saturates".  Cases that either side rejects as not exactly representable are skipped.
+    rng = np.random.default_rng(20240114)
+    ran = 0
+    variants = set()
+    for trial in range(120):
+        M, N = int(rng.integers(1, 200)), int(rng.integers(1, 150))
+        K = int(rng.choice([1, 5, 16, 31, 48, 100, 160, 333]))
+        E = int(rng.integers(3, 7))
+        Mb = int(rng.choice([2, 3, 4, 6, 7, 8, 10, 12]))
+        rounding = int(rng.integers(0, 2))
+        flags = int(rng.integers(0, 2))
+        b_prod = 2 ** E - 18 + int(rng.integers(-3, 8))
+        b_acc = b_prod - int(rng.integers(0, 4))
+        Mp = Mb if rng.random() < 0.7 else int(rng.choice([3, 5, 7, 9]))
+        prod = LbaFormat(Mp, E, b_prod, rounding, flags)
+        acc = LbaFormat(Mb, E, b_acc, rounding, flags)
+        order = SEQ if rng.random() < 0.4 else CHK
+        chunk = int(rng.choice([16, 16, 32, 7, 48]))
+        scale = float(rng.choice([0.02, 1.0, 30.0, 120.0]))
+        A = synth.e4m3_encode(synth.gaussian((M, K), 7000 + trial) * scale)
+        B = synth.e4m3_encode(synth.gaussian((N, K), 8000 + trial) * scale)
+        if rng.random() < 0.3:
+            A, B = A & 0x7F, B & 0x7F                      # same-sign products: the sums run into saturation
+        sa = torch.tensor([float(rng.uniform(0.5, 2.0))])
+        sb = torch.linspace(0.5, 1.5, N)
+        try:
+            want = ref_gemm(A, B, sa, sb, None, prod, acc, order, chunk)
+        except orc.OracleError:
+            continue
+        try:
+            plan = lba.describe_plan(M, N, K, prod, acc, order, chunk)
+            got = gpu_gemm(A, B, sa, sb, None, prod, acc, order, chunk)
+        except lba.LbaError as e:
+            assert e.status == -3                          # format not carried exactly: refused, never approximated
+            continue
+        assert_bit_equal(got, want, f"trial {trial}: {M}x{N}x{K} {prod} {acc} order {order}/{chunk} scale {scale} [{plan}]")
+        variants.add((plan.split("q=")[1].split()[0], plan.split("order=")[1].split()[0]))
+        ran += 1
+    assert ran >= 60, ran
+    assert len(variants) >= 8, variants
+
+
 def test_zero_and_empty_shapes():
     prod, acc = code_domain_formats(7, 4)
     one = torch.ones(1)
