@@ -327,6 +327,31 @@ def test_conv2d_matches_direct_convolution(case, name):
         assert_bit_equal(got, want, f"{case} {name} {order}/{chunk}")
 
 
+def test_random_convolution_geometries():
+    rng = np.random.default_rng(424242)
+    for trial in range(40):
+        B, H, W = int(rng.integers(1, 4)), int(rng.integers(3, 20)), int(rng.integers(3, 20))
+        Cin = int(rng.choice([1, 3, 5, 16, 24, 32, 48]))
+        Cout = int(rng.integers(1, 90))
+        KH, KW = int(rng.integers(1, 6)), int(rng.integers(1, 6))
+        stride = (int(rng.integers(1, 4)), int(rng.integers(1, 4)))
+        pad = (int(rng.integers(0, 3)), int(rng.integers(0, 3)))
+        if H + 2 * pad[0] < KH or W + 2 * pad[1] < KW:
+            continue
+        name = ["m7e4_code", "m4e4", "m7e4_code_rne"][trial % 3]
+        prod, acc = FORMATS[name]
+        x = synth.e4m3_encode(synth.gaussian((B, H, W, Cin), 9000 + trial).relu() * 60.0)
+        w = synth.e4m3_encode(synth.gaussian((Cout, KH, KW, Cin), 9500 + trial) * 60.0)
+        sx = torch.tensor([0.7])
+        sw = torch.linspace(0.5, 2.0, Cout)
+        order, chunk = [(CHK, 16), (SEQ, 16), (CHK, 32), (CHK, 5)][trial % 4]
+        got = lba.lba_conv2d(x.to(DEV), w.to(DEV), sx.to(DEV), sw.to(DEV), None, stride, pad, prod, acc, order, chunk)
+        want = orc.conv2d(x.numpy(), w.numpy(), sx.numpy(), sw.numpy(), None, stride, pad, prod.as_tuple(),
+                          acc.as_tuple(), order, chunk)
+        assert tuple(got.shape) == want.shape
+        assert_bit_equal(got, want, f"trial {trial}: B{B} {H}x{W}x{Cin}->{Cout} k{KH}x{KW} s{stride} p{pad} {name} {order}/{chunk}")
+
+
 @pytest.mark.parametrize("tile", [0, 1, 2, 3])
 def test_conv2d_every_tile(tile):
     prod, acc = code_domain_formats(7, 4)
