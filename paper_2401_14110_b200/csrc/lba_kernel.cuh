@@ -1,30 +1,32 @@
-// LBA contraction kernel for sm_100a: out[m][n] = epilogue(chain_k FMAq(A[m][k], B[n][k], .)).
+// LBA contraction kernels for sm_100a: out[m][n] = epilogue(chain_k FMAq(A[m][k], B[n][k], .)).
 //
-// The method rounds after every single addition (Eq. 4 of the paper), so no group of products
-// may be summed exactly first: tensor cores are excluded by definition and the kernel is bound
-// by CUDA-core issue slots.  Everything below exists to keep the per-MAC instruction count low.
+// The method rounds after every single addition (Eq. 4 of the paper), so no group of products may be summed
+// exactly first: tensor-core MMA is excluded by definition and the kernels are bound by CUDA-core issue slots
+// and pipes.  Everything below exists to keep the per-MAC instruction count low.
 //
-// Carrier arithmetic.  Values are carried in binary32 registers, scaled by a power of two so that
-// the format's underflow threshold R_UF sits at binary32's smallest normal 2^-126:
-//   * product:   p' = x' * w' with x' = x * 2^sx, w' = w * 2^sw, sx + sw = b_prod - 126.  The
-//     product of two E4M3 values has at most 8 significant bits, so it is exact; `mul.ftz` then
-//     flushes exactly the products with |x*w| < R_UF_prod (Eq. 2, second case).
-//   * sum:       t = fma.rz.ftz(p', 2^(b_acc-b_prod), S').  The FMA forms p'*c + S' exactly and
-//     rounds once toward zero to 24 bits; cutting a toward-zero result to M < 24 bits again toward
-//     zero equals cutting the exact sum (truncations compose), so `t & mask` is the floor of Eq. 2
-//     on the exact sum.  `.ftz` flushes exactly the sums below R_UF_acc, because a toward-zero
-//     rounding never moves a value across 2^-126.
+// Carrier arithmetic.  Values are carried in binary32 registers, scaled by a power of two so that the
+// format's underflow threshold R_UF sits at binary32's smallest normal 2^-126:
+//   * product:   p' = x' * w' with x' = x * 2^sx, w' = w * 2^sw, sx + sw = b_prod - 126.  The product of two
+//     E4M3 values has at most 8 significant bits, so it is exact; `mul.ftz` then flushes exactly the products
+//     with |x*w| < R_UF_prod (Eq. 2, second case).
+//   * sum:       t = fma.rz.ftz(p', 2^(b_acc-b_prod), S').  The FMA forms p'*c + S' exactly and rounds once
+//     toward zero to 24 bits; cutting a toward-zero result to M < 24 bits again toward zero equals cutting the
+//     exact sum (truncations compose), so `t & mask` is the floor of Eq. 2 on the exact sum.  `.ftz` flushes
+//     exactly the sums below R_UF_acc, because a toward-zero rounding never moves a value across 2^-126.
 //   * saturation: min.xorsign.abs(t, R_OF') = sign(t) * min(|t|, R_OF'), one instruction.
-// That is 4 instructions per emulated MAC (FMUL, FFMA, LOP3, FMNMX) when Q_prod can neither round
-// nor saturate (M_prod >= 7 and 448^2 < R_OF_prod), which the host proves per call.
-// Nearest-even does not compose with a binary32 rounding, so that mode first builds the
-// round-to-odd value of the exact sum (from the FMA rounded down and up) and rounds that.
+// Nearest-even does not compose with a binary32 rounding, so that mode first builds the round-to-odd image of
+// the exact sum (from directed roundings of the FMA) and rounds that.
+// The host proves per call which branches of Eq. 2 E4M3 inputs can reach and picks the cheapest exact variant.
 //
-// Data path.  A CTA owns a BM x BN output tile and walks K in slabs of 16 bytes per row: each
-// thread fetches 16-byte row pieces (one 128-bit load), decodes the 16 E4M3 bytes to scaled
-// binary32 once, and stores them k-major into shared memory (double buffered, one barrier per
-// slab).  Each thread keeps a TM x TN register micro-tile of running sums and walks k in order;
-// K is never split across threads, so the paper's accumulation order is kept by construction.
+// Two kernels share the operand loaders:
+//   lba_contract_packed_kernel  packed f32x2 arithmetic (two outputs per instruction), the magnitude clamp
+//                               skipped per slab under a norm bound; floor and nearest-even; the fast path
+//   lba_contract_kernel         scalar arithmetic, always clamped; any chunk length, 24-bit accumulator
+// Data path of both: a CTA owns a BM x BN output tile and walks K in slabs of 16 bytes per row; each thread
+// fetches 16-byte row pieces (one 128-bit load), decodes the 16 E4M3 bytes to scaled binary32 once, and stores
+// them k-major into shared memory (double buffered, one barrier per slab).  Each thread keeps a TM x TN
+// register micro-tile of running sums and walks k in order; K is never split across threads, so the paper's
+// accumulation order is kept by construction.
 #pragma once
 #include <cstdint>
 #include <type_traits>
