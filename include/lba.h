@@ -100,6 +100,17 @@ int lba_gemm_batched(const uint8_t* A, const uint8_t* B, const float* scale_a, i
                      int64_t stride_a, int64_t stride_b, int64_t stride_out, const lba_fmt* prod_fmt,
                      const lba_fmt* acc_fmt, int order, int chunk, float* out, void* stream);
 
+/* Re-computation for the recursive overflow straight-through estimator (Sec. 4 and App. D): the forward pass is
+ * deterministic, so the backward pass can replay it instead of storing one bit per FMAq.  For every output
+ * (m, n), in SEQUENTIAL order, last[m][n] is the largest step index i with
+ *     | Q_prod(x_i w_i) + S_i | >= R_OF(acc_fmt)        (STE^OF = 0 at that step),
+ * or -1 if the accumulator never overflowed: the recursive estimator cuts the gradient of every product before
+ * that step and passes the later ones, so this index is all it needs per output (App. D).
+ *   A, B   device, as for lba_gemm; formats must use floor rounding (else LBA_ERR_FORMAT)
+ *   last   device, [M][N] int32 */
+int lba_gemm_last_overflow(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt,
+                           const lba_fmt* acc_fmt, int32_t* last, void* stream);
+
 /* Convolution as an implicit GEMM (Eq. 3 with m = (b, oh, ow), n = c_out and k walking
  * (kh, kw, c_in), c_in fastest).  Padded taps are the value 0 and still count toward the
  * chunk position.  Dilation 1, groups 1.

@@ -89,3 +89,18 @@ def dot(prod_fmt, acc_fmt, order, chunk, xcodes, wcodes) -> Fraction:
             c = fmaq(prod_fmt, acc_fmt, x, w, c)
         total = quantise(acc_fmt, c + total)
     return total
+
+
+def last_overflow(prod_fmt, acc_fmt, xcodes, wcodes) -> int:
+    """Sequential order: index of the last step with |Q_prod(x w) + S| >= R_OF(acc) (where the overflow
+    straight-through estimator of App. D is 0), or -1."""
+    M, E, b, _, _ = acc_fmt
+    top = r_of(M, E, b)
+    s = Fraction(0)
+    last = -1
+    for i, (xc, wc) in enumerate(zip(xcodes, wcodes)):
+        t = quantise(prod_fmt, decode_e4m3(int(xc)) * decode_e4m3(int(wc))) + s
+        if abs(t) >= top:
+            last = i
+        s = quantise(acc_fmt, t)
+    return last

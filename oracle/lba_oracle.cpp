@@ -260,9 +260,12 @@ struct Chain {
   Dy second;       // running sum over finished chunks
   int64_t in_chunk;
   int status;
+  int64_t steps;          // FMAq steps taken so far
+  int64_t last_overflow;  // index of the last step with |Q_prod(x w) + S| >= R_OF(acc), or -1 (STE^OF of App. D)
 
   Chain(const Fmt* p, const Fmt* a, int ord, int64_t ch)
-      : prod(p), acc(a), order(ord), chunk(ch), first(kZero), second(kZero), in_chunk(0), status(LBO_OK) {}
+      : prod(p), acc(a), order(ord), chunk(ch), first(kZero), second(kZero), in_chunk(0), status(LBO_OK), steps(0),
+        last_overflow(-1) {}
 
   void close_chunk() {
     Dy sum;
@@ -279,6 +282,8 @@ struct Chain {
     Dy p = quantise(*prod, mul_exact(x, w));
     Dy sum;
     if (!add_exact(p, first, &sum)) { status = LBO_ERR_RANGE; return; }
+    if (sum.mag != 0 && cmp_mag(sum, acc->r_of) >= 0) last_overflow = steps;
+    ++steps;
     first = quantise(*acc, sum);
   }
 
@@ -520,6 +525,28 @@ int lbo_gemm(const uint8_t* A, const uint8_t* B, const float* sa, int sa_len, co
     for (int64_t n = 0; n < N; ++n) {
       int s = gemm_point(g, m, n, out + m * N + n);
       if (s != LBO_OK) return s;
+    }
+    return (int)LBO_OK;
+  });
+}
+
+// last[M][N]: for the SEQUENTIAL chain of every output, the index of the last step whose exact sum
+// Q_prod(x_i w_i) + S_i reached R_OF of the accumulator format (the step where STE^OF of App. D is 0), or -1
+int lbo_gemm_last_overflow(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, int64_t K, const lbo_fmt* pf,
+                           const lbo_fmt* af, int32_t* last, int nthreads) {
+  GemmArgs g;
+  const float one = 1.0f;
+  int st = fill_gemm(&g, A, B, &one, 1, &one, 1, nullptr, M, N, K, pf, af, LBO_ORDER_SEQUENTIAL, 1);
+  if (st != LBO_OK) return st;
+  if (!last && M * N > 0) return LBO_ERR_ARG;
+  return parallel_items(M, nthreads, [&](int64_t m) {
+    for (int64_t n = 0; n < N; ++n) {
+      Chain c(&g.prod, &g.acc, g.order, g.chunk);
+      for (int64_t i = 0; i < K; ++i) {
+        c.push(A[m * K + i], B[n * K + i]);
+        if (c.status != LBO_OK) return c.status;
+      }
+      last[m * N + n] = (int32_t)c.last_overflow;
     }
     return (int)LBO_OK;
   });

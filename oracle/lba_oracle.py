@@ -156,6 +156,19 @@ def gemm_points(A, B, scale_a, scale_b, bias, prod_fmt, acc_fmt, order, chunk, m
     return out
 
 
+def gemm_last_overflow(A, B, prod_fmt, acc_fmt, nthreads=0):
+    """int32 [M][N]: last sequential step at which the input of Q_acc reached R_OF (STE^OF = 0, App. D), -1 if none."""
+    A, Ap = _u8(A)
+    B, Bp = _u8(B)
+    M, K = A.shape
+    N, _ = B.shape
+    pf, af = _fmt(prod_fmt), _fmt(acc_fmt)
+    out = np.empty((M, N), dtype=np.int32)
+    _check(lib().lbo_gemm_last_overflow(Ap, Bp, C.c_int64(M), C.c_int64(N), C.c_int64(K), C.byref(pf), C.byref(af),
+                                        out.ctypes.data_as(C.POINTER(C.c_int32)), C.c_int(nthreads or default_threads())))
+    return out
+
+
 def conv_out_hw(H, W, KH, KW, stride, pad):
     sh, sw = stride
     ph, pw = pad

@@ -14,7 +14,7 @@ from .formats import LbaFormat, ORDER_CHUNKED, PAPER_CHUNK
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liblba.so")
 
-EXPORTS = ["lba_gemm", "lba_gemm_batched", "lba_conv2d", "lba_gemm_host_workspace_bytes", "lba_gemm_host",
+EXPORTS = ["lba_gemm", "lba_gemm_batched", "lba_gemm_last_overflow", "lba_conv2d", "lba_gemm_host_workspace_bytes", "lba_gemm_host",
            "lba_conv2d_host_workspace_bytes", "lba_conv2d_host", "lba_gemm_host_static", "lba_count_nan_codes", "lba_describe_plan",
            "lba_set_tile_override", "lba_device_error", "lba_status_string", "lba_last_cuda_error", "lba_version"]
 
@@ -53,6 +53,8 @@ def load_library():
                  C.c_int64, C.POINTER(_Fmt), C.POINTER(_Fmt), C.c_int, C.c_int, C.c_void_p]
     lib.lba_gemm.argtypes = gemm_args + [C.c_void_p]
     lib.lba_gemm_host.argtypes = gemm_args + [C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.lba_gemm_last_overflow.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.POINTER(_Fmt),
+                                           C.POINTER(_Fmt), C.c_void_p, C.c_void_p]
     lib.lba_gemm_batched.argtypes = gemm_args[:7] + [C.c_int64] * 7 + gemm_args[10:] + [C.c_void_p]
     lib.lba_gemm_host_static.argtypes = gemm_args + [C.c_void_p]
     conv_args = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p] + [C.c_int] * 11 + \
@@ -146,6 +148,21 @@ def lba_gemm_batched(A, B, scale_a, scale_b, bias, prod_fmt, acc_fmt, order=ORDE
                                 _dev(scale_b, torch.float32, "scale_b"), scale_b.numel(),
                                 _dev(bias, torch.float32, "bias"), Z, M, N, K, M * K, stride_b, M * N, C.byref(pf),
                                 C.byref(af), order, chunk, _dev(out, torch.float32, "out"), _stream(stream)))
+    return out
+
+
+def lba_gemm_last_overflow(A, B, prod_fmt, acc_fmt, out=None, stream=None):
+    """int32 [M][N]: index of the last sequential step at which Q_acc overflowed, -1 if none.  See lba.h."""
+    lib = load_library()
+    M, K = A.shape
+    N, K2 = B.shape
+    if K != K2:
+        raise ValueError("A and B disagree on K")
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.int32, device=A.device)
+    pf, af = _fmt(prod_fmt), _fmt(acc_fmt)
+    _check(lib.lba_gemm_last_overflow(_dev(A, torch.uint8, "A"), _dev(B, torch.uint8, "B"), M, N, K, C.byref(pf),
+                                      C.byref(af), _dev(out, torch.int32, "last"), _stream(stream)))
     return out
 
 

@@ -22,6 +22,7 @@ LBA_DECL(QM_RNE_WIDE, ORD_SEQ) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_SLAB) LBA_DECL(QM
 
 cudaError_t launch_umma_family(int load, const Problem& p, cudaStream_t stream);
 cudaError_t read_umma_error(int* code);
+cudaError_t launch_last_overflow(int load, const Problem& p, cudaStream_t stream);
 
 namespace {
 
@@ -409,6 +410,31 @@ int lba_gemm_batched(const uint8_t* A, const uint8_t* B, const float* scale_a, i
     if ((st = run(q, pl, vec ? LD_GEMM_VEC : LD_ANY, (cudaStream_t)stream)) != LBA_OK) return st;
   }
   return LBA_OK;
+}
+
+int lba_gemm_last_overflow(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt,
+                           const lba_fmt* acc_fmt, int32_t* last, void* stream) {
+  if (M < 0 || N < 0 || K < 0 || K > 2147483647LL) return LBA_ERR_SHAPE;
+  Plan pl;
+  const int st = make_plan(prod_fmt, acc_fmt, LBA_ORDER_SEQUENTIAL, 1, K, &pl);
+  if (st != LBA_OK) return st;
+  if (pl.qm != QM_FLOOR_FAST && pl.qm != QM_FLOOR_FULL) return LBA_ERR_FORMAT;  // floor rounding only
+  if (M == 0 || N == 0) return LBA_OK;
+  if (!last || (K > 0 && (!A || !B))) return LBA_ERR_NULL;
+  if ((N + 63) / 64 > 65535) return LBA_ERR_SHAPE;
+  Problem p;
+  std::memset(&p, 0, sizeof(p));
+  p.M = M;
+  p.N = N;
+  p.K = K;
+  p.batch = 1;
+  p.A = A;
+  p.B = B;
+  p.out = reinterpret_cast<float*>(last);
+  apply_plan(&p, pl);
+  const bool vec = K % BK == 0 && aligned16(A) && aligned16(B);
+  const cudaError_t e = launch_last_overflow(vec ? LD_GEMM_VEC : LD_ANY, p, (cudaStream_t)stream);
+  return e == cudaSuccess ? LBA_OK : cuda_fail(e);
 }
 
 int lba_conv2d(const uint8_t* x, const uint8_t* w, const float* scale_x, int scale_x_len, const float* scale_w,

@@ -299,8 +299,12 @@ struct RowLoader {
 };
 
 // ------------------------------------------------------------------ the kernel
-template <int BM, int BN, int TM, int TN, int QM, int ORD, int LD>
+// TRACK (floor quantisers, sequential order): instead of the sums, write for every output the index of the
+// last step whose exact sum Q_prod(x_i w_i) + S_i reached R_OF, or -1 (the "last overflow" that the recursive
+// overflow straight-through estimator of App. D needs); `out` is then read as int32 [M][N].
+template <int BM, int BN, int TM, int TN, int QM, int ORD, int LD, bool TRACK = false>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(const Problem p) {
+  static_assert(!TRACK || (QM == QM_FLOOR_FULL && ORD == ORD_SEQ), "tracking variant");
   constexpr int NT = (BM / TM) * (BN / TN);
   constexpr int TX = BN / TN;
   constexpr int ROWS = BM + BN;
@@ -367,6 +371,15 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
       }
   };
 
+  int last[TRACK ? TM : 1][TRACK ? TN : 1];
+  if (TRACK) {
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+      for (int j = 0; j < TN; ++j) last[TRACK ? i : 0][TRACK ? j : 0] = -1;
+  }
+  int kbase = 0;  // TRACK: global index of the slab's first step
+
   auto mac_step = [&](int buf, int kk) {
     float a[TM], b[TN];
 #pragma unroll
@@ -382,7 +395,17 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
 #pragma unroll
     for (int i = 0; i < TM; ++i)
 #pragma unroll
-      for (int j = 0; j < TN; ++j) acc1[i][j] = q_acc_fma<QM>(q_prod<QM>(a[i], b[j], qp), cc, acc1[i][j], qa);
+      for (int j = 0; j < TN; ++j) {
+        if (TRACK) {
+          // the exact sum reaches R_OF exactly when its toward-zero image cut to M bits does (R_OF is on that
+          // grid); zero-padded steps past K are not steps of the chain and are not counted
+          const float t = and_bits(fma_rz_ftz(q_prod<QM>(a[i], b[j], qp), cc, acc1[i][j]), qa.mask);
+          if (fabsf(t) >= qa.sat && kbase + kk < (int)K) last[TRACK ? i : 0][TRACK ? j : 0] = kbase + kk;
+          acc1[i][j] = clamp_mag(t, qa.sat);
+        } else {
+          acc1[i][j] = q_acc_fma<QM>(q_prod<QM>(a[i], b[j], qp), cc, acc1[i][j], qa);
+        }
+      }
   };
 
   // ---- main loop
@@ -419,9 +442,25 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
     }
     if (s + 1 < nslab) decode_store(raw, buf ^ 1);
     __syncthreads();
+    kbase += BK;
   }
   if (ORD == ORD_CHUNK_SLAB && slabs_in_chunk > 0) close_chunk();
   if (ORD == ORD_CHUNK_ANY && k_in_chunk > 0) close_chunk();
+
+  if (TRACK) {
+    int* const lastz = reinterpret_cast<int*>(p.out) + (int64_t)blockIdx.z * p.batch_out;
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+      const int64_t m = m0 + (i / 4) * (BM / 2) + ty * 4 + (i % 4);
+      if (m >= p.M) continue;
+#pragma unroll
+      for (int j = 0; j < TN; ++j) {
+        const int64_t n = n0 + (j / 4) * (BN / 2) + tx * 4 + (j % 4);
+        if (n < p.N) lastz[m * p.N + n] = last[TRACK ? i : 0][TRACK ? j : 0];
+      }
+    }
+    return;
+  }
 
   // ---- epilogue: back to real values, +0 for every zero, scales and bias in binary32
   float* const outz = p.out + (int64_t)blockIdx.z * p.batch_out;

@@ -194,3 +194,39 @@ def test_planted_mistakes_are_caught_by_the_pins():
     assert chain(lambda v: ex.quantise(prod, v), lambda v: ex.quantise((7, 4, 10, 1, 1), v), 4) != Fraction(63.5)
     # last product dropped (the S_{N-1} misprint of Eq. 8-9)
     assert chain(lambda v: ex.quantise(prod, v), lambda v: ex.quantise(acc, v), 4) != good
+
+
+def test_last_overflow_index_hand_worked_and_against_exact_rationals():
+    # chain A of the golden file: x = w = 4.0, products saturate Q_prod to 15.9375; the accumulator input is
+    # 15.9375, 31.875, 47.8125, 63.6875 (all below R_OF_acc = 63.75), then 63.5 + 15.9375 = 79.4375 >= 63.75 at
+    # step 4 and at every later step (S stays at 63.75)
+    prod, acc = (7, 4, 12, 0, 1), (7, 4, 10, 0, 1)
+    for K, want in ((1, -1), (4, -1), (5, 4), (7, 6)):
+        x = np.full((1, K), 0x48, np.uint8)
+        assert orc.gemm_last_overflow(x, x, prod, acc)[0, 0] == want
+        assert ex.last_overflow(prod, acc, x[0], x[0]) == want
+    # a negative tail brings the sum back below R_OF: the last overflow stays where it was
+    x = np.array([[0x48] * 6 + [0xC8] * 3], np.uint8)      # six times +4, three times -4
+    w = np.full((1, 9), 0x48, np.uint8)
+    assert orc.gemm_last_overflow(x, w, prod, acc)[0, 0] == 5
+    # a step that adds nothing while S sits at R_OF still has |0 + S| >= R_OF
+    x = np.array([[0x48] * 6 + [0x00] * 2], np.uint8)
+    assert orc.gemm_last_overflow(x, np.full((1, 8), 0x48, np.uint8), prod, acc)[0, 0] == 7
+    # random small cases against the exact-rational restatement of Eq. 2 / Eq. 4
+    rng = np.random.default_rng(5)
+    finite = np.array([c for c in range(256) if (c & 0x7F) != 0x7F], np.uint8)
+    hits = 0
+    for trial in range(60):
+        K = int(rng.integers(1, 40))
+        A = finite[rng.integers(0, finite.size, (3, K))]
+        B = finite[rng.integers(0, finite.size, (2, K))]
+        if trial % 2:
+            A, B = A & 0x7F, B & 0x7F
+        fm = [((7, 4, 12, 0, 1), (7, 4, 10, 0, 1)), ((7, 4, -2, 0, 1), (7, 4, -4, 0, 1)), ((4, 4, 0, 0, 0), (5, 4, 2, 0, 0))][trial % 3]
+        got = orc.gemm_last_overflow(A, B, fm[0], fm[1])
+        for m in range(3):
+            for n in range(2):
+                want = ex.last_overflow(fm[0], fm[1], A[m], B[n])
+                assert got[m, n] == want
+                hits += want >= 0
+    assert hits > 20
