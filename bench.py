@@ -44,6 +44,19 @@ ISSUE_SLOTS_PER_MAC_LEVEL1 = 2.0
 ISSUE_SLOTS_PER_CHUNK_CLOSE = 2.5
 
 
+# DRAM bytes (read + write) of ONE launch of the dominant kernel, from the ncu captures summarised under profiles/
+# (workload, kernel description) -> (bytes, what was captured).  A kernel that is not listed reports null.
+NCU_DRAM_TRAFFIC = {
+    ("resnet18_fwd_conv_stack_b32_224_m7e4_chunk16", "tile=64x64x16 micro=4x8 q=floor_fast order=chunk16 load=conv_vec"):
+        (3425280, "one of the 14 launches (layer2.0.conv2, M=25088 N=128 K=1152): 3.4 MB read, 0 written while the kernel "
+                  "ran (its 12.8 MB output was still in L2); algorithmic 16.2 MB"),
+    ("single_lba_gemm_8192x8192x1024_m7e4_chunk16", "tile=64x64x16 micro=4x8 q=floor_fast order=chunk16 load=gemm_vec"):
+        (230230528, "16.9 MB read + 213.3 MB written; algorithmic 272 MB (part of the output still in L2)"),
+    ("single_lba_gemm_8192x8192x1024_m7e4_sequential", "tile=128x128x16 micro=8x8 q=floor_fast order=seq load=gemm_vec"):
+        (229131776, "17.0 MB read + 212.1 MB written; algorithmic 272 MB (part of the output still in L2)"),
+}
+
+
 def issue_slots_per_mac(order_chunked: bool, chunk: int) -> float:
     return ISSUE_SLOTS_PER_MAC_LEVEL1 + (ISSUE_SLOTS_PER_CHUNK_CLOSE / chunk if order_chunked else 0.0)
 
@@ -364,7 +377,8 @@ def main():
     achieved = dom["macs"] / (dom["ms"] * 1e-3) / 1e9
     roofline = {
         "bound": "alu", "achieved": achieved, "peak": peak, "unit": UNIT, "frac": achieved / peak,
-        "traffic": None,
+        "traffic": NCU_DRAM_TRAFFIC.get((WORKLOAD, dom_key), (None, None))[0],
+        "traffic_note": NCU_DRAM_TRAFFIC.get((WORKLOAD, dom_key), (None, "no ncu capture of this kernel on this workload"))[1],
         "kernel": dom_key, "kernel_launches_per_step": dom["launches"], "kernel_ms_per_step": dom["ms"],
         "kernel_share_of_step": dom["ms"] / sum(per_call_ms),
         "peak_derivation": f"{sm_count} SMs x {ISSUE_LANES_PER_SM_CLK} lanes issued per clock x {max_mhz:.0f} MHz "
