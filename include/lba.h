@@ -111,6 +111,30 @@ int lba_gemm_batched(const uint8_t* A, const uint8_t* B, const float* scale_a, i
 int lba_gemm_last_overflow(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt,
                            const lba_fmt* acc_fmt, int32_t* last, void* stream);
 
+/* Straight-through estimators of App. D, per FMAq step. */
+enum { LBA_STE_OF = 1, LBA_STE_DIFF = 2 };
+
+/* Re-computation for the fine-grained estimators (Sec. 4, App. D): replays the chain of every output (m, n) in the
+ * given order and writes one bit per FMAq step, 1 where the estimator passes the gradient:
+ *   LBA_STE_OF    1 iff | Q_prod(x_i w_i) + S_i | < R_OF(acc_fmt)
+ *   LBA_STE_DIFF  1 iff | FMAq(x_i, w_i, S_i) - S_i | > eps2 * ( |x_i w_i| + eps1 ), evaluated in binary32 with one
+ *                 rounding (to nearest) per operation: the subtraction, the addition, the multiplication;
+ *                 eps1, eps2 > 0 are given in the domain of the decoded code values (the paper does not print
+ *                 the values it used).
+ * mask1 [M][N][ceil(K/32)] uint32: bit (i % 32) of word (i / 32) belongs to step i of the first hierarchy (the only
+ * one in sequential order).  In chunked order mask2 [M][N][ceil(C/32)], C = ceil(K/chunk), holds in the same way the
+ * bits of the steps T <- Q_acc(C_j + T) that fold chunk j into the second hierarchy, with the chunk sum C_j in the
+ * product's place; a single chunk (chunk >= K) still has its one fold.  Unused high bits of a last word are 0.
+ * The "immediate" estimators use the bits as they are; the "recursive" ones pass a product's gradient only if every
+ * later step on its path to the output passed, which the caller derives from the same bits (App. D).
+ *   A, B          device, as for lba_gemm; floor rounding only (else LBA_ERR_FORMAT)
+ *   ste           LBA_STE_OF or LBA_STE_DIFF (else LBA_ERR_ORDER); eps1, eps2 are read for LBA_STE_DIFF only, and
+ *                 values for which the comparison cannot be carried in binary32 give LBA_ERR_FORMAT
+ *   mask1, mask2  device, written in full by the call; mask2 may be NULL in sequential order */
+int lba_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt,
+                      const lba_fmt* acc_fmt, int order, int chunk, int ste, float eps1, float eps2, uint32_t* mask1,
+                      uint32_t* mask2, void* stream);
+
 /* Convolution as an implicit GEMM (Eq. 3 with m = (b, oh, ow), n = c_out and k walking
  * (kh, kw, c_in), c_in fastest).  Padded taps are the value 0 and still count toward the
  * chunk position.  Dilation 1, groups 1.

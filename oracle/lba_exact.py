@@ -104,3 +104,39 @@ def last_overflow(prod_fmt, acc_fmt, xcodes, wcodes) -> int:
             last = i
         s = quantise(acc_fmt, t)
     return last
+
+
+def ste_bits(prod_fmt, acc_fmt, order, chunk, xcodes, wcodes, kind, eps1=0.0, eps2=0.0):
+    """STE value of every FMAq step (App. D), as two lists of 0/1: the steps of the first hierarchy and, in
+    chunked order (order = 1), the folds of the chunk sums.  kind "OF": 1 iff |term + S| < R_OF(acc).
+    kind "DIFF": 1 iff |z - S| > eps2 * (|u| + eps1), u the unquantised product (the chunk sum at a fold), every
+    operation (the subtraction, the addition, the multiplication) rounded to binary32."""
+    import numpy as np
+    M, E, b, _, _ = acc_fmt
+    top = r_of(M, E, b)
+
+    def ste(term, u, s):
+        z = quantise(acc_fmt, term + s)
+        if kind == "OF":
+            return z, int(abs(term + s) < top)
+        den = np.float32(np.float32(float(abs(u))) + np.float32(eps1))
+        thr = np.float32(np.float32(eps2) * den)
+        d = np.float32(float(z)) - np.float32(float(s))      # z and S are binary32 numbers; one rounded subtraction
+        return z, int(abs(d) > thr)
+
+    first, second = [], []
+    s = t = Fraction(0)
+    n_in = 0
+    for xc, wc in zip(xcodes, wcodes):
+        xw = decode_e4m3(int(xc)) * decode_e4m3(int(wc))
+        s, bit = ste(quantise(prod_fmt, xw), xw, s)
+        first.append(bit)
+        n_in += 1
+        if order == 1 and n_in == chunk:
+            t, bit = ste(s, s, t)
+            second.append(bit)
+            s, n_in = Fraction(0), 0
+    if order == 1 and n_in > 0:
+        t, bit = ste(s, s, t)
+        second.append(bit)
+    return first, second

@@ -72,6 +72,7 @@ enum {
 };
 
 enum { LBO_ORDER_SEQUENTIAL = 0, LBO_ORDER_CHUNKED = 1 };
+enum { LBO_STE_NONE = 0, LBO_STE_OF = 1, LBO_STE_DIFF = 2 };  // straight-through estimators of App. D
 
 }  // extern "C"
 
@@ -262,29 +263,57 @@ struct Chain {
   int status;
   int64_t steps;          // FMAq steps taken so far
   int64_t last_overflow;  // index of the last step with |Q_prod(x w) + S| >= R_OF(acc), or -1 (STE^OF of App. D)
+  // straight-through estimators of App. D, evaluated for the step just taken (first hierarchy) and for
+  // the chunk just folded (second hierarchy, where the chunk sum stands in for the product)
+  int ste_kind;           // LBO_STE_NONE / LBO_STE_OF / LBO_STE_DIFF
+  float eps1, eps2;       // DIFF only
+  int ste_first, ste_second;
+  int64_t chunks_closed;
 
   Chain(const Fmt* p, const Fmt* a, int ord, int64_t ch)
       : prod(p), acc(a), order(ord), chunk(ch), first(kZero), second(kZero), in_chunk(0), status(LBO_OK), steps(0),
-        last_overflow(-1) {}
+        last_overflow(-1), ste_kind(0), eps1(0.0f), eps2(0.0f), ste_first(0), ste_second(0), chunks_closed(0) {}
+
+  // STE^OF: 1 iff |term + S| < R_OF.   STE^DIFF: 1 iff |z - S| / (|u| + eps1) > eps2, u the unquantised product
+  // (the chunk sum at the second hierarchy); the DIFF comparison is taken in binary32, round to nearest:
+  // |fl(z - S)| > fl(eps2 * fl(|u| + eps1)).
+  int ste(const Dy& exact_sum, const Dy& z, const Dy& s_before, const Dy& u) {
+    if (ste_kind == LBO_STE_OF) return !(exact_sum.mag != 0 && cmp_mag(exact_sum, acc->r_of) >= 0);
+    if (ste_kind == LBO_STE_DIFF) {
+      float zf, sf, uf;
+      if (!to_float(z, &zf) || !to_float(s_before, &sf) || !to_float(u, &uf)) { status = LBO_ERR_RANGE; return 0; }
+      volatile float d = zf - sf;   // one binary32 subtraction (exact whenever the difference fits 24 bits)
+      volatile float den = std::fabs(uf) + eps1;
+      volatile float thr = eps2 * den;
+      return std::fabs(d) > thr;
+    }
+    return 0;
+  }
 
   void close_chunk() {
     Dy sum;
     if (!add_exact(first, second, &sum)) { status = LBO_ERR_RANGE; return; }
-    second = quantise(*acc, sum);
+    Dy t = quantise(*acc, sum);
+    if (ste_kind) ste_second = ste(sum, t, second, first);
+    second = t;
     first = kZero;
     in_chunk = 0;
+    ++chunks_closed;
   }
 
   // one FMAq step: first <- Q_acc(Q_prod(x*w) + first)
   void fmaq_step(uint8_t xcode, uint8_t wcode) {
     Dy x, w;
     if (!decode_e4m3(xcode, &x) || !decode_e4m3(wcode, &w)) { status = LBO_ERR_NAN_CODE; return; }
-    Dy p = quantise(*prod, mul_exact(x, w));
+    Dy xw = mul_exact(x, w);
+    Dy p = quantise(*prod, xw);
     Dy sum;
     if (!add_exact(p, first, &sum)) { status = LBO_ERR_RANGE; return; }
     if (sum.mag != 0 && cmp_mag(sum, acc->r_of) >= 0) last_overflow = steps;
     ++steps;
-    first = quantise(*acc, sum);
+    Dy z = quantise(*acc, sum);
+    if (ste_kind) ste_first = ste(sum, z, first, xw);
+    first = z;
   }
 
   // in chunked order, a full chunk is folded into the second hierarchy
@@ -547,6 +576,52 @@ int lbo_gemm_last_overflow(const uint8_t* A, const uint8_t* B, int64_t M, int64_
         if (c.status != LBO_OK) return c.status;
       }
       last[m * N + n] = (int32_t)c.last_overflow;
+    }
+    return (int)LBO_OK;
+  });
+}
+
+// STE bit masks of the re-computation pass (Sec. 4, App. D).  mask1[M][N][ceil(K/32)]: bit (i % 32) of word i / 32
+// is the STE value of step i of the first hierarchy (of the only one in sequential order).  mask2[M][N][ceil(C/32)],
+// C = ceil(K / chunk), chunked order only: the same for the step that folds chunk j into the second hierarchy.
+// Unused high bits of the last word are 0.
+int lbo_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, int64_t K, const lbo_fmt* pf,
+                      const lbo_fmt* af, int order, int64_t chunk, int kind, float eps1, float eps2, uint32_t* mask1,
+                      uint32_t* mask2, int nthreads) {
+  GemmArgs g;
+  const float one = 1.0f;
+  int st = fill_gemm(&g, A, B, &one, 1, &one, 1, nullptr, M, N, K, pf, af, order, chunk);
+  if (st != LBO_OK) return st;
+  if (kind != LBO_STE_OF && kind != LBO_STE_DIFF) return LBO_ERR_ARG;
+  if (kind == LBO_STE_DIFF && !(eps1 > 0.0f && eps2 > 0.0f)) return LBO_ERR_ARG;
+  const bool chunked = order == LBO_ORDER_CHUNKED;
+  const int64_t W1 = (K + 31) / 32;
+  const int64_t C = chunked ? (K + chunk - 1) / chunk : 0;
+  const int64_t W2 = (C + 31) / 32;
+  if ((M * N * W1 > 0 && !mask1) || (M * N * W2 > 0 && !mask2)) return LBO_ERR_ARG;
+  return parallel_items(M, nthreads, [&](int64_t m) {
+    for (int64_t n = 0; n < N; ++n) {
+      uint32_t* w1 = mask1 + (m * N + n) * W1;
+      uint32_t* w2 = chunked ? mask2 + (m * N + n) * W2 : nullptr;
+      for (int64_t i = 0; i < W1; ++i) w1[i] = 0;
+      for (int64_t i = 0; i < W2; ++i) w2[i] = 0;
+      Chain c(&g.prod, &g.acc, g.order, g.chunk);
+      c.ste_kind = kind;
+      c.eps1 = eps1;
+      c.eps2 = eps2;
+      for (int64_t i = 0; i < K; ++i) {
+        c.fmaq_step(A[m * K + i], B[n * K + i]);
+        if (c.status != LBO_OK) return c.status;
+        if (c.ste_first) w1[i / 32] |= 1u << (i % 32);
+        const int64_t before = c.chunks_closed;
+        c.end_of_step();
+        if (c.status != LBO_OK) return c.status;
+        if (c.chunks_closed != before && c.ste_second) w2[before / 32] |= 1u << (before % 32);
+      }
+      const int64_t before = c.chunks_closed;
+      c.finish();   // folds a short last chunk
+      if (c.status != LBO_OK) return c.status;
+      if (c.chunks_closed != before && c.ste_second) w2[before / 32] |= 1u << (before % 32);
     }
     return (int)LBO_OK;
   });

@@ -14,7 +14,7 @@ from .formats import LbaFormat, ORDER_CHUNKED, PAPER_CHUNK
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liblba.so")
 
-EXPORTS = ["lba_gemm", "lba_gemm_batched", "lba_gemm_last_overflow", "lba_conv2d", "lba_gemm_host_workspace_bytes", "lba_gemm_host",
+EXPORTS = ["lba_gemm", "lba_gemm_batched", "lba_gemm_last_overflow", "lba_gemm_ste_mask", "lba_conv2d", "lba_gemm_host_workspace_bytes", "lba_gemm_host",
            "lba_conv2d_host_workspace_bytes", "lba_conv2d_host", "lba_gemm_host_static", "lba_count_nan_codes", "lba_describe_plan",
            "lba_set_tile_override", "lba_device_error", "lba_status_string", "lba_last_cuda_error", "lba_version"]
 
@@ -55,6 +55,9 @@ def load_library():
     lib.lba_gemm_host.argtypes = gemm_args + [C.c_void_p, C.c_size_t, C.c_void_p]
     lib.lba_gemm_last_overflow.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.POINTER(_Fmt),
                                            C.POINTER(_Fmt), C.c_void_p, C.c_void_p]
+    lib.lba_gemm_ste_mask.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.POINTER(_Fmt),
+                                      C.POINTER(_Fmt), C.c_int, C.c_int, C.c_int, C.c_float, C.c_float, C.c_void_p,
+                                      C.c_void_p, C.c_void_p]
     lib.lba_gemm_batched.argtypes = gemm_args[:7] + [C.c_int64] * 7 + gemm_args[10:] + [C.c_void_p]
     lib.lba_gemm_host_static.argtypes = gemm_args + [C.c_void_p]
     conv_args = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p] + [C.c_int] * 11 + \
@@ -164,6 +167,29 @@ def lba_gemm_last_overflow(A, B, prod_fmt, acc_fmt, out=None, stream=None):
     _check(lib.lba_gemm_last_overflow(_dev(A, torch.uint8, "A"), _dev(B, torch.uint8, "B"), M, N, K, C.byref(pf),
                                       C.byref(af), _dev(out, torch.int32, "last"), _stream(stream)))
     return out
+
+
+STE_OF, STE_DIFF = 1, 2
+
+
+def lba_gemm_ste_mask(A, B, prod_fmt, acc_fmt, order=ORDER_CHUNKED, chunk=PAPER_CHUNK, ste=STE_OF, eps1=0.0, eps2=0.0,
+                      stream=None):
+    """(mask1 int32 [M][N][ceil(K/32)], mask2 int32 [M][N][ceil(ceil(K/chunk)/32)] or None): one STE bit per FMAq
+    step, as 32-bit words (torch has no unsigned 32-bit arithmetic; the bit patterns are what counts).  See lba.h."""
+    lib = load_library()
+    M, K = A.shape
+    N, K2 = B.shape
+    if K != K2:
+        raise ValueError("A and B disagree on K")
+    mask1 = torch.empty((M, N, (K + 31) // 32), dtype=torch.int32, device=A.device)
+    mask2 = None
+    if order == ORDER_CHUNKED:
+        mask2 = torch.empty((M, N, ((K + chunk - 1) // max(chunk, 1) + 31) // 32), dtype=torch.int32, device=A.device)
+    pf, af = _fmt(prod_fmt), _fmt(acc_fmt)
+    _check(lib.lba_gemm_ste_mask(_dev(A, torch.uint8, "A"), _dev(B, torch.uint8, "B"), M, N, K, C.byref(pf), C.byref(af),
+                                 order, chunk, ste, C.c_float(eps1), C.c_float(eps2), _dev(mask1, torch.int32, "mask1"),
+                                 None if mask2 is None else _dev(mask2, torch.int32, "mask2"), _stream(stream)))
+    return mask1, mask2
 
 
 def lba_conv2d(x, w, scale_x, scale_w, bias, stride, pad, prod_fmt, acc_fmt, order=ORDER_CHUNKED, chunk=PAPER_CHUNK,

@@ -23,6 +23,7 @@ LBA_DECL(QM_RNE_WIDE, ORD_SEQ) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_SLAB) LBA_DECL(QM
 cudaError_t launch_umma_family(int load, const Problem& p, cudaStream_t stream);
 cudaError_t read_umma_error(int* code);
 cudaError_t launch_last_overflow(int load, const Problem& p, cudaStream_t stream);
+cudaError_t launch_ste_mask(int ord, int diff, int load, const Problem& p, cudaStream_t stream);
 
 namespace {
 
@@ -63,6 +64,8 @@ struct Plan {
   float rne_k_acc, rne_k_prod;
   QConst qp, qa;
   int chunk_slabs, chunk;
+  int kp, ka, sx;   // product carrier = value * 2^kp, accumulator carrier = value * 2^ka, A operand = x * 2^sx
+  double a_top;     // largest reachable accumulator magnitude (real domain)
 };
 
 bool fmt_ok(const lba_fmt* f) {
@@ -146,6 +149,10 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
 
   const int sx = (kp >= 0) ? kp / 2 : -((-kp + 1) / 2);  // floor(kp / 2)
   const int sw = kp - sx;
+  pl->kp = kp;
+  pl->ka = ka;
+  pl->sx = sx;
+  pl->a_top = a_sat ? a_rof : max_sum;
   pl->dec_a = (float)std::ldexp(1.0, 120 + sx);
   pl->dec_b = (float)std::ldexp(1.0, 120 + sw);
   pl->c = (float)std::ldexp(1.0, ka - kp);
@@ -434,6 +441,71 @@ int lba_gemm_last_overflow(const uint8_t* A, const uint8_t* B, int64_t M, int64_
   apply_plan(&p, pl);
   const bool vec = K % BK == 0 && aligned16(A) && aligned16(B);
   const cudaError_t e = launch_last_overflow(vec ? LD_GEMM_VEC : LD_ANY, p, (cudaStream_t)stream);
+  return e == cudaSuccess ? LBA_OK : cuda_fail(e);
+}
+
+int lba_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt,
+                      const lba_fmt* acc_fmt, int order, int chunk, int ste, float eps1, float eps2, uint32_t* mask1,
+                      uint32_t* mask2, void* stream) {
+  if (M < 0 || N < 0 || K < 0 || K > 2147483647LL - 64) return LBA_ERR_SHAPE;
+  if (ste != LBA_STE_OF && ste != LBA_STE_DIFF) return LBA_ERR_ORDER;
+  Plan pl;
+  const int st = make_plan(prod_fmt, acc_fmt, order, chunk, K, &pl);
+  if (st != LBA_OK) return st;
+  if (pl.qm != QM_FLOOR_FAST && pl.qm != QM_FLOOR_FULL) return LBA_ERR_FORMAT;  // floor rounding only
+  const bool chunked = order == LBA_ORDER_CHUNKED;
+  const int64_t chunks = chunked ? (K + chunk - 1) / chunk : 0;
+  Problem p;
+  std::memset(&p, 0, sizeof(p));
+  if (ste == LBA_STE_DIFF) {
+    // the comparison |z - S| > fl(eps2 * fl(|u| + eps1)) runs on values scaled by 2^kd relative to the real
+    // domain; scaling by a power of two commutes with binary32 rounding as long as nothing leaves the normal
+    // range on either side, which is checked here for the extreme operands
+    if (!(eps1 > 0.0f) || !(eps2 > 0.0f) || !std::isfinite(eps1) || !std::isfinite(eps2)) return LBA_ERR_FORMAT;
+    const int kd = pl.ka + 32;
+    const auto normal = [kd](double v) {  // a normal binary32 magnitude in the real domain and after scaling
+      const double lo = std::ldexp(1.0, -126), hi = std::ldexp(1.0, 127), w = std::ldexp(v, kd);
+      return v >= lo && v < hi && w >= lo && w < hi;
+    };
+    const double u_max = std::fmax(std::ldexp(1.0, 18), pl.a_top);   // |x w| < 2^18; a chunk sum <= a_top
+    const double u_min = std::ldexp(1.0, -18);                       // smallest non-zero |x w| and chunk sum
+    // smallest non-zero |z - S|: one step of the accumulator's grid in its lowest binade
+    const bool a_flush = (acc_fmt->flags & LBA_FLAG_UNDERFLOW) && acc_fmt->bias < 18;
+    const double d_min = a_flush ? std::ldexp(1.0, -acc_fmt->bias - acc_fmt->man_bits) : u_min;
+    for (const double v : {(double)eps1, u_max + eps1, (double)eps2 * eps1, (double)eps2 * (u_max + eps1), u_min, u_max,
+                           d_min, 2.0 * pl.a_top})
+      if (!normal(v)) return LBA_ERR_FORMAT;
+    // A is rescaled so that A' * B' = |x w| * 2^kd; |x| lies in [2^-9, 448]
+    const int sa = pl.sx + kd - pl.kp;
+    if (sa - 9 < -126 || sa + 9 > 127) return LBA_ERR_FORMAT;
+    const int kp = pl.kp;
+    p.diff_scale = std::ldexp(1.0f, 32);
+    p.diff_a_scale = std::ldexp(1.0f, kd - kp);
+    p.diff_eps1 = std::ldexp(eps1, kd);
+    p.diff_eps2 = eps2;
+  }
+  if (M == 0 || N == 0 || K == 0) return LBA_OK;
+  if (!A || !B || !mask1 || (chunked && !mask2)) return LBA_ERR_NULL;
+  if ((N + 63) / 64 > 65535) return LBA_ERR_SHAPE;
+  p.M = M;
+  p.N = N;
+  p.K = K;
+  p.batch = 1;
+  p.A = A;
+  p.B = B;
+  apply_plan(&p, pl);
+  p.mask1 = mask1;
+  p.mask2 = mask2;
+  p.mask2_words = (chunks + 31) / 32;
+  // the single-chunk shortcut of the forward pass does not apply: the fold of that one chunk is a step too
+  int ord = ORD_SEQ;
+  if (chunked) {
+    ord = chunk % BK == 0 ? ORD_CHUNK_SLAB : ORD_CHUNK_ANY;
+    p.chunk = chunk;
+    p.chunk_slabs = chunk / BK;
+  }
+  const bool vec = K % BK == 0 && aligned16(A) && aligned16(B);
+  const cudaError_t e = launch_ste_mask(ord, ste == LBA_STE_DIFF, vec ? LD_GEMM_VEC : LD_ANY, p, (cudaStream_t)stream);
   return e == cudaSuccess ? LBA_OK : cuda_fail(e);
 }
 

@@ -75,6 +75,15 @@ struct Problem {
   int pq;              // PackedProd: what Q_prod does beyond the flush
   int rne_packed;      // nearest-even: 1 if the packed kernel's exponent headroom suffices
   float rne_k_acc, rne_k_prod;  // 1.5 * 2^(23 - M) for the accumulator and the product format
+  // straight-through-estimator masks (tracking variants of the scalar kernel only)
+  uint32_t *mask1, *mask2;
+  int64_t mask2_words;  // ceil(chunks / 32)
+  // DIFF comparison: carried in "accumulator carrier * diff_scale" so that differences of neighbouring
+  // accumulator values stay normal numbers
+  float diff_scale;    // accumulator carrier -> comparison scaling (2^32)
+  float diff_a_scale;  // product-carrier A operand -> operand whose product with B is |x w| in comparison scaling
+  float diff_eps1;     // eps1 in comparison scaling
+  float diff_eps2;     // eps2 (a pure ratio)
 };
 
 // ------------------------------------------------------------------ scalar building blocks
@@ -299,12 +308,24 @@ struct RowLoader {
 };
 
 // ------------------------------------------------------------------ the kernel
-// TRACK (floor quantisers, sequential order): instead of the sums, write for every output the index of the
-// last step whose exact sum Q_prod(x_i w_i) + S_i reached R_OF, or -1 (the "last overflow" that the recursive
-// overflow straight-through estimator of App. D needs); `out` is then read as int32 [M][N].
-template <int BM, int BN, int TM, int TN, int QM, int ORD, int LD, bool TRACK = false>
+// TRACK selects the re-computation passes of the straight-through estimators (Sec. 4, App. D; floor quantisers
+// only).  Instead of the sums the kernel then writes what the backward pass needs:
+//   TRACK_LAST_OF  sequential order; `out` is read as int32 [M][N]: index of the last step whose exact sum
+//                  Q_prod(x_i w_i) + S_i reached R_OF, or -1 (all the recursive overflow estimator needs);
+//   TRACK_MASK_OF  one bit per FMAq step, 1 iff |Q_prod(x_i w_i) + S_i| < R_OF (STE^OF);
+//   TRACK_MASK_DIFF one bit per FMAq step, 1 iff |z - S| > eps2 * (|x_i w_i| + eps1) (STE^DIFF), each of the three
+//                  operations rounded to binary32.
+// Masks: mask1 uint32 [M][N][ceil(K/32)], bit i%32 of word i/32 for step i; in chunked order mask2
+// [M][N][ceil(chunks/32)] holds the bits of the folds T <- Q_acc(C + T), the chunk sum C in the product's place.
+enum { TRACK_NONE = 0, TRACK_LAST_OF = 1, TRACK_MASK_OF = 2, TRACK_MASK_DIFF = 3 };
+
+template <int BM, int BN, int TM, int TN, int QM, int ORD, int LD, int TRACK = TRACK_NONE>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(const Problem p) {
-  static_assert(!TRACK || (QM == QM_FLOOR_FULL && ORD == ORD_SEQ), "tracking variant");
+  static_assert(TRACK == TRACK_NONE || QM == QM_FLOOR_FULL, "tracking variants use the floor quantisers");
+  static_assert(TRACK != TRACK_LAST_OF || ORD == ORD_SEQ, "last-overflow index: sequential order");
+  static_assert(TRACK == TRACK_NONE || ORD != ORD_CHUNK16, "tracking variants: generic orders");
+  constexpr bool MASKS = TRACK == TRACK_MASK_OF || TRACK == TRACK_MASK_DIFF;
+  constexpr bool DIFF = TRACK == TRACK_MASK_DIFF;
   constexpr int NT = (BM / TM) * (BN / TN);
   constexpr int TX = BN / TN;
   constexpr int ROWS = BM + BN;
@@ -360,25 +381,83 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
   const float cc = p.c;
   const QConst qp = p.qp, qa = p.qa;
 
+  // ---- tracking state
+  constexpr bool LAST = TRACK == TRACK_LAST_OF;
+  int last[LAST ? TM : 1][LAST ? TN : 1];                       // TRACK_LAST_OF
+  uint32_t bits1[MASKS ? TM : 1][MASKS ? TN : 1];               // current word of mask1
+  uint32_t bits2[MASKS && CHUNKED ? TM : 1][MASKS && CHUNKED ? TN : 1];
+  float prev1[DIFF ? TM : 1][DIFF ? TN : 1];                    // S and T in the comparison's scaling
+  float prev2[DIFF && CHUNKED ? TM : 1][DIFF && CHUNKED ? TN : 1];
+#pragma unroll
+  for (int i = 0; i < TM; ++i)
+#pragma unroll
+    for (int j = 0; j < TN; ++j) {
+      if (LAST) last[LAST ? i : 0][LAST ? j : 0] = -1;
+      if (MASKS) bits1[MASKS ? i : 0][MASKS ? j : 0] = 0u;
+      if (MASKS && CHUNKED) bits2[MASKS && CHUNKED ? i : 0][MASKS && CHUNKED ? j : 0] = 0u;
+      if (DIFF) prev1[DIFF ? i : 0][DIFF ? j : 0] = 0.0f;
+      if (DIFF && CHUNKED) prev2[DIFF && CHUNKED ? i : 0][DIFF && CHUNKED ? j : 0] = 0.0f;
+    }
+  int kbase = 0;     // global index of the slab's first step
+  int chunk_id = 0;  // index of the chunk being accumulated
+  uint32_t* const mask1z = MASKS ? p.mask1 : nullptr;
+  uint32_t* const mask2z = MASKS ? p.mask2 : nullptr;
+  const int64_t W1 = MASKS ? (K + 31) / 32 : 0;
+  const int64_t W2 = MASKS ? p.mask2_words : 0;
+  const float dscale = p.diff_scale, deps1 = p.diff_eps1, deps2 = p.diff_eps2;
+
+  // one word of a mask for every output of the thread
+  auto flush_words = [&](uint32_t* base, int64_t words, int64_t w, auto& bits) {
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+      const int64_t m = m0 + (i / 4) * (BM / 2) + ty * 4 + (i % 4);
+#pragma unroll
+      for (int j = 0; j < TN; ++j) {
+        const int64_t n = n0 + (j / 4) * (BN / 2) + tx * 4 + (j % 4);
+        if (m < p.M && n < p.N) base[(m * p.N + n) * words + w] = bits[i][j];
+        bits[i][j] = 0u;
+      }
+    }
+  };
+
+  // STE bit of one step: t = the exact sum cut toward zero to M bits (|t| >= R_OF exactly when the exact
+  // sum is), z = Q_acc of it, u = the unquantised product or the chunk sum (DIFF scaling), s_prev = S before
+  auto ste_bit = [&](float t, float z, float u, float& s_prev) -> uint32_t {
+    if (DIFF) {
+      const float zd = mul_ieee(z, dscale);                       // exact: z is a normal number
+      const float d = fabsf(__fadd_rn(zd, -s_prev));              // one rounding, as the definition says
+      s_prev = zd;
+      const float thr = __fmul_rn(deps2, __fadd_rn(fabsf(u), deps1));
+      return d > thr ? 1u : 0u;
+    }
+    (void)z; (void)u; (void)s_prev;
+    return fabsf(t) < qa.sat ? 1u : 0u;
+  };
+
   auto close_chunk = [&]() {  // second hierarchy: T <- Q_acc(C + T), C <- 0
 #pragma unroll
     for (int i = 0; i < TM; ++i)
 #pragma unroll
       for (int j = 0; j < TN; ++j) {
         float& t2 = acc2[CHUNKED ? i : 0][CHUNKED ? j : 0];
-        t2 = q_acc_fma<QM>(acc1[i][j], 1.0f, t2, qa);
+        if (MASKS && CHUNKED) {
+          const float t = and_bits(fma_rz_ftz(acc1[i][j], 1.0f, t2), qa.mask);
+          const float z = clamp_mag(t, qa.sat);
+          const float u = DIFF ? mul_ieee(acc1[i][j], dscale) : 0.0f;
+          bits2[MASKS && CHUNKED ? i : 0][MASKS && CHUNKED ? j : 0] |=
+              ste_bit(t, z, u, prev2[DIFF && CHUNKED ? i : 0][DIFF && CHUNKED ? j : 0]) << (chunk_id & 31);
+          t2 = z;
+          if (DIFF) prev1[DIFF ? i : 0][DIFF ? j : 0] = 0.0f;
+        } else {
+          t2 = q_acc_fma<QM>(acc1[i][j], 1.0f, t2, qa);
+        }
         acc1[i][j] = 0.0f;
       }
+    if constexpr (MASKS && CHUNKED) {
+      if ((chunk_id & 31) == 31) flush_words(mask2z, W2, (int64_t)(chunk_id >> 5), bits2);
+      ++chunk_id;
+    }
   };
-
-  int last[TRACK ? TM : 1][TRACK ? TN : 1];
-  if (TRACK) {
-#pragma unroll
-    for (int i = 0; i < TM; ++i)
-#pragma unroll
-      for (int j = 0; j < TN; ++j) last[TRACK ? i : 0][TRACK ? j : 0] = -1;
-  }
-  int kbase = 0;  // TRACK: global index of the slab's first step
 
   auto mac_step = [&](int buf, int kk) {
     float a[TM], b[TN];
@@ -392,16 +471,29 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
       const float4 v = *reinterpret_cast<const float4*>(&Bs[buf][kk][h * (BN / 2) + tx * 4]);
       b[h * 4 + 0] = v.x; b[h * 4 + 1] = v.y; b[h * 4 + 2] = v.z; b[h * 4 + 3] = v.w;
     }
+    float ad[DIFF ? TM : 1];
+    if (DIFF) {
+#pragma unroll
+      for (int i = 0; i < TM; ++i) ad[DIFF ? i : 0] = mul_ieee(a[i], p.diff_a_scale);
+    }
 #pragma unroll
     for (int i = 0; i < TM; ++i)
 #pragma unroll
       for (int j = 0; j < TN; ++j) {
-        if (TRACK) {
+        if (TRACK != TRACK_NONE) {
           // the exact sum reaches R_OF exactly when its toward-zero image cut to M bits does (R_OF is on that
-          // grid); zero-padded steps past K are not steps of the chain and are not counted
+          // grid); zero-padded steps past K are not steps of the chain: no index, bit 0
           const float t = and_bits(fma_rz_ftz(q_prod<QM>(a[i], b[j], qp), cc, acc1[i][j]), qa.mask);
-          if (fabsf(t) >= qa.sat && kbase + kk < (int)K) last[TRACK ? i : 0][TRACK ? j : 0] = kbase + kk;
-          acc1[i][j] = clamp_mag(t, qa.sat);
+          const float z = clamp_mag(t, qa.sat);
+          const bool real_step = kbase + kk < (int)K;
+          if (LAST) {
+            if (fabsf(t) >= qa.sat && real_step) last[LAST ? i : 0][LAST ? j : 0] = kbase + kk;
+          } else {
+            const float u = DIFF ? mul_ieee(ad[DIFF ? i : 0], b[j]) : 0.0f;  // exact |x w| in the comparison's scaling
+            const uint32_t bit = ste_bit(t, z, u, prev1[DIFF ? i : 0][DIFF ? j : 0]);
+            bits1[MASKS ? i : 0][MASKS ? j : 0] |= (real_step ? bit : 0u) << ((kbase + kk) & 31);
+          }
+          acc1[i][j] = z;
         } else {
           acc1[i][j] = q_acc_fma<QM>(q_prod<QM>(a[i], b[j], qp), cc, acc1[i][j], qa);
         }
@@ -440,6 +532,9 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
         }
       }
     }
+    if constexpr (MASKS) {  // a word of mask1 is complete after every second slab
+      if ((s & 1) || s + 1 == nslab) flush_words(mask1z, W1, (int64_t)(s >> 1), bits1);
+    }
     if (s + 1 < nslab) decode_store(raw, buf ^ 1);
     __syncthreads();
     kbase += BK;
@@ -447,7 +542,13 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
   if (ORD == ORD_CHUNK_SLAB && slabs_in_chunk > 0) close_chunk();
   if (ORD == ORD_CHUNK_ANY && k_in_chunk > 0) close_chunk();
 
-  if (TRACK) {
+  if constexpr (MASKS) {
+    if constexpr (CHUNKED) {
+      if ((chunk_id & 31) != 0) flush_words(mask2z, W2, (int64_t)(chunk_id >> 5), bits2);
+    }
+    return;
+  }
+  if (LAST) {
     int* const lastz = reinterpret_cast<int*>(p.out) + (int64_t)blockIdx.z * p.batch_out;
 #pragma unroll
     for (int i = 0; i < TM; ++i) {
@@ -456,7 +557,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
 #pragma unroll
       for (int j = 0; j < TN; ++j) {
         const int64_t n = n0 + (j / 4) * (BN / 2) + tx * 4 + (j % 4);
-        if (n < p.N) lastz[m * p.N + n] = last[TRACK ? i : 0][TRACK ? j : 0];
+        if (n < p.N) lastz[m * p.N + n] = last[LAST ? i : 0][LAST ? j : 0];
       }
     }
     return;

@@ -328,6 +328,76 @@ def test_last_overflow_index_edge_cases():
     assert lba.device_error() == 0
 
 
+STE_ORDERS = [(SEQ, 1), (CHK, 16), (CHK, 32), (CHK, 5), (CHK, 4096)]
+
+
+def _u32(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_paper", "m4e4", "m10e5", "m4e3_mnist", "m7e4_no_uf"])
+@pytest.mark.parametrize("ste", ["of", "diff"])
+def test_ste_masks_match_oracle(name, ste):
+    # one bit per FMAq step (App. D): first hierarchy and, in chunked order, the folds of the chunk sums
+    prod, acc = FORMATS[name]
+    kind, e1, e2 = (lba.STE_OF, 0.0, 0.0) if ste == "of" else (lba.STE_DIFF, 2.0 ** -20, 0.25)
+    zeros = ones = zeros2 = 0
+    for (M, N, K) in ((1, 1, 1), (70, 45, 37), (66, 67, 160), (33, 129, 1000)):
+        for regime in (0, 1, 2, 3):
+            A, B = _overflow_case(M, N, K, regime, 100 * regime + K + 7)
+            for order, chunk in STE_ORDERS:
+                g1, g2 = lba.lba_gemm_ste_mask(A.to(DEV), B.to(DEV), prod, acc, order, chunk, kind, e1, e2)
+                w1, w2 = orc.gemm_ste_mask(A.numpy(), B.numpy(), prod.as_tuple(), acc.as_tuple(), order, chunk,
+                                           orc.STE_OF if ste == "of" else orc.STE_DIFF, e1, e2)
+                what = f"{name} {ste} {M}x{N}x{K} regime {regime} order {order} chunk {chunk}"
+                bad = np.argwhere(_u32(g1) != w1)
+                assert bad.size == 0, f"{what}: mask1 differs in {len(bad)} words, first at {bad[0]}"
+                assert (g2 is None) == (w2 is None)
+                if w2 is not None:
+                    bad = np.argwhere(_u32(g2) != w2)
+                    assert bad.size == 0, f"{what}: mask2 differs in {len(bad)} words, first at {bad[0]}"
+                    zeros2 += int(w2.size * 32 - np.unpackbits(w2.view(np.uint8)).sum())
+                n1 = int(np.unpackbits(w1.view(np.uint8)).sum())
+                ones += n1
+                zeros += M * N * K - n1
+    assert ones > 10000 and zeros > 10000 and zeros2 > 0
+
+
+def test_ste_mask_edge_cases():
+    prod, acc = M7E4_PAPER
+    x = torch.full((1, 7), 0x48, dtype=torch.uint8, device=DEV)
+    m1, m2 = lba.lba_gemm_ste_mask(x, x, prod, acc, SEQ, 1, lba.STE_OF)
+    assert m2 is None and int(m1[0, 0, 0]) == 0b0001111            # hand-worked: four steps stay below 63.75
+    m1, m2 = lba.lba_gemm_ste_mask(x, x, prod, acc, CHK, 16, lba.STE_OF)
+    assert int(m1[0, 0, 0]) == 0b0001111 and int(m2[0, 0, 0]) == 0  # the one chunk's fold sees 63.75 = R_OF
+    # stagnation at 32: the difference estimator stops passing once the product is swamped
+    a = torch.full((1, 300), 0x30, dtype=torch.uint8, device=DEV)
+    w = torch.full((1, 300), 0x28, dtype=torch.uint8, device=DEV)
+    m1, _ = lba.lba_gemm_ste_mask(a, w, prod, acc, SEQ, 1, lba.STE_DIFF, 1e-6, 0.5)
+    assert [int(v) & 0xFFFFFFFF for v in m1[0, 0]] == [0xFFFFFFFF] * 8 + [0, 0]
+    # empty problems, K = 0
+    e1, e2 = lba.lba_gemm_ste_mask(torch.empty((3, 0), dtype=torch.uint8, device=DEV),
+                                   torch.empty((2, 0), dtype=torch.uint8, device=DEV), prod, acc, CHK, 16, lba.STE_OF)
+    assert e1.shape == (3, 2, 0) and e2.shape == (3, 2, 0)
+    # odd base pointers: byte-wise loader
+    Abig = (synth.random_codes((40 * 64 + 3,), 3) & 0x7F).to(DEV)
+    Bbig = (synth.random_codes((33 * 64 + 5,), 4) & 0x7F).to(DEV)
+    A, B = Abig[3:].view(40, 64), Bbig[5:].view(33, 64)
+    g1, g2 = lba.lba_gemm_ste_mask(A, B, prod, acc, CHK, 16, lba.STE_DIFF, 1e-4, 0.5)
+    w1, w2 = orc.gemm_ste_mask(A.cpu().numpy(), B.cpu().numpy(), prod.as_tuple(), acc.as_tuple(), CHK, 16,
+                               orc.STE_DIFF, 1e-4, 0.5)
+    assert (_u32(g1) == w1).all() and (_u32(g2) == w2).all()
+    # rejected arguments
+    with pytest.raises(lba.LbaError):
+        lba.lba_gemm_ste_mask(A, B, *FORMATS["m7e4_code_rne"], CHK, 16, lba.STE_OF)
+    with pytest.raises(lba.LbaError):
+        lba.lba_gemm_ste_mask(A, B, prod, acc, CHK, 16, 7)
+    with pytest.raises(lba.LbaError):
+        lba.lba_gemm_ste_mask(A, B, prod, acc, CHK, 16, lba.STE_DIFF, 0.0, 0.5)
+    with pytest.raises(lba.LbaError):
+        lba.lba_gemm_ste_mask(A, B, prod, acc, CHK, 16, lba.STE_DIFF, 1e-45, 0.5)
+
+
 def test_zero_and_empty_shapes():
     prod, acc = code_domain_formats(7, 4)
     one = torch.ones(1)

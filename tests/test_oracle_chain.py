@@ -230,3 +230,75 @@ def test_last_overflow_index_hand_worked_and_against_exact_rationals():
                 assert got[m, n] == want
                 hits += want >= 0
     assert hits > 20
+
+
+def _bits_of(words, n):
+    return [(int(words[i // 32]) >> (i % 32)) & 1 for i in range(n)]
+
+
+def test_ste_masks_hand_worked_chains():
+    prod, acc = (7, 4, 12, 0, 1), (7, 4, 10, 0, 1)
+    # x = w = 4.0: the accumulator input is 15.9375, 31.875, 47.8125, 63.6875, then 79.4375 and 79.6875... >= 63.75:
+    # STE^OF passes the first four steps only
+    x = np.full((1, 7), 0x48, np.uint8)
+    m1, m2 = orc.gemm_ste_mask(x, x, prod, acc, 0, 1, orc.STE_OF)
+    assert m2 is None and m1.shape == (1, 1, 1) and m1[0, 0, 0] == 0b0001111
+    # the stagnation chain (x = 0.5, w = 0.25, product 0.125): every step adds 0.125 exactly until S = 32, where
+    # the grid step is 0.25 and the product is swamped: z - S = 0.125 = |x w| for 256 steps, then 0.  STE^DIFF with
+    # eps2 = 0.5 therefore passes exactly the first 256 steps; nothing ever overflows, so STE^OF passes all 300
+    a = np.full((1, 300), 0x30, np.uint8)
+    w = np.full((1, 300), 0x28, np.uint8)
+    m1, _ = orc.gemm_ste_mask(a, w, prod, acc, 0, 1, orc.STE_DIFF, 1e-6, 0.5)
+    assert _bits_of(m1[0, 0], 300) == [1] * 256 + [0] * 44
+    assert (m1[0, 0, 9] >> 12) == 0                                   # unused high bits of the last word
+    m1, _ = orc.gemm_ste_mask(a, w, prod, acc, 0, 1, orc.STE_OF)
+    assert _bits_of(m1[0, 0], 300) == [1] * 300
+    # chunks of 16 keep every first-level sum at <= 2.0 and the folds add 2.0 to T <= 37.5 exactly: all bits pass
+    m1, m2 = orc.gemm_ste_mask(a, w, prod, acc, 1, 16, orc.STE_DIFF, 1e-6, 0.5)
+    assert _bits_of(m1[0, 0], 300) == [1] * 300 and _bits_of(m2[0, 0], 19) == [1] * 19 and m2.shape == (1, 1, 1)
+    # K = 576 in chunks of 16: T climbs by 2.0 per fold and saturates at 63.75 at the 32nd fold (exact sum 64):
+    # STE^OF of the folds is 1 for folds 0..30 and 0 from fold 31 on
+    a = np.full((1, 576), 0x30, np.uint8)
+    w = np.full((1, 576), 0x28, np.uint8)
+    m1, m2 = orc.gemm_ste_mask(a, w, prod, acc, 1, 16, orc.STE_OF)
+    assert _bits_of(m2[0, 0], 36) == [1] * 31 + [0] * 5 and m2.shape == (1, 1, 2)
+    assert all(v == 0xFFFFFFFF for v in m1[0, 0])
+    # a single chunk still has its fold: x = w = 4.0, K = 7, chunk 16: C = 63.75 (saturated), |C + 0| >= R_OF
+    x = np.full((1, 7), 0x48, np.uint8)
+    m1, m2 = orc.gemm_ste_mask(x, x, prod, acc, 1, 16, orc.STE_OF)
+    assert m1[0, 0, 0] == 0b0001111 and m2[0, 0, 0] == 0
+    # a zero product never passes STE^DIFF (App. D sets alpha = 0 there): z = S
+    x = np.array([[0x48, 0x00, 0x48]], np.uint8)
+    m1, _ = orc.gemm_ste_mask(x, np.full((1, 3), 0x48, np.uint8), prod, acc, 0, 1, orc.STE_DIFF, 1e-6, 0.01)
+    assert m1[0, 0, 0] == 0b101
+
+
+def test_ste_masks_against_exact_rationals_and_last_overflow():
+    rng = np.random.default_rng(11)
+    finite = np.array([c for c in range(256) if (c & 0x7F) != 0x7F], np.uint8)
+    fmts = [((7, 4, 12, 0, 1), (7, 4, 10, 0, 1)), ((7, 4, -2, 0, 1), (7, 4, -4, 0, 1)), ((4, 4, 0, 0, 0), (5, 4, 2, 0, 0)),
+            ((4, 3, 5, 0, 1), (4, 3, 5, 0, 1))]
+    zeros = ones = 0
+    for trial in range(48):
+        K = int(rng.integers(1, 90))
+        A = finite[rng.integers(0, finite.size, (2, K))]
+        B = finite[rng.integers(0, finite.size, (2, K))]
+        if trial % 2:
+            A, B = A & 0x7F, B & 0x7F
+        pf, af = fmts[trial % 4]
+        order, chunk = [(0, 1), (1, 16), (1, 5), (1, 32), (1, 100)][trial % 5]
+        for kind, name, e1, e2 in ((orc.STE_OF, "OF", 0.0, 0.0), (orc.STE_DIFF, "DIFF", 2.0 ** -20, 0.25),
+                                   (orc.STE_DIFF, "DIFF", 1e-3, 0.9)):
+            m1, m2 = orc.gemm_ste_mask(A, B, pf, af, order, chunk, kind, e1, e2)
+            for m in range(2):
+                for n in range(2):
+                    f, s = ex.ste_bits(pf, af, order, chunk, A[m], B[n], name, e1, e2)
+                    assert _bits_of(m1[m, n], K) == f
+                    assert order == 0 or _bits_of(m2[m, n], len(s)) == s
+                    zeros += f.count(0)
+                    ones += f.count(1)
+                    if kind == orc.STE_OF and order == 0:
+                        # the last-overflow index is the position of the highest 0 bit of the sequential OF mask
+                        want = max((i for i, b in enumerate(f) if b == 0), default=-1)
+                        assert orc.gemm_last_overflow(A[m:m + 1], B[n:n + 1], pf, af)[0, 0] == want
+    assert zeros > 500 and ones > 500
