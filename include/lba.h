@@ -121,8 +121,10 @@ enum { LBA_STE_OF = 1, LBA_STE_DIFF = 2 };
  *                 rounding (to nearest) per operation: the subtraction, the addition, the multiplication;
  *                 eps1, eps2 > 0 are given in the domain of the decoded code values (the paper does not print
  *                 the values it used).
- * mask1 [M][N][ceil(K/32)] uint32: bit (i % 32) of word (i / 32) belongs to step i of the first hierarchy (the only
- * one in sequential order).  In chunked order mask2 [M][N][ceil(C/32)], C = ceil(K/chunk), holds in the same way the
+ * mask1 [M][ceil(K/32)][N] uint32 (the words of one step range lie side by side for neighbouring n, which is how
+ * both this kernel and a gradient GEMM that reduces over n touch them): bit (i % 32) of word (i / 32) of output
+ * (m, n) belongs to step i of the first hierarchy (the only one in sequential order).  In chunked order
+ * mask2 [M][ceil(C/32)][N], C = ceil(K/chunk), holds in the same way the
  * bits of the steps T <- Q_acc(C_j + T) that fold chunk j into the second hierarchy, with the chunk sum C_j in the
  * product's place; a single chunk (chunk >= K) still has its one fold.  Unused high bits of a last word are 0.
  * The "immediate" estimators use the bits as they are; the "recursive" ones pass a product's gradient only if every

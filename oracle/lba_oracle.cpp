@@ -581,10 +581,10 @@ int lbo_gemm_last_overflow(const uint8_t* A, const uint8_t* B, int64_t M, int64_
   });
 }
 
-// STE bit masks of the re-computation pass (Sec. 4, App. D).  mask1[M][N][ceil(K/32)]: bit (i % 32) of word i / 32
-// is the STE value of step i of the first hierarchy (of the only one in sequential order).  mask2[M][N][ceil(C/32)],
-// C = ceil(K / chunk), chunked order only: the same for the step that folds chunk j into the second hierarchy.
-// Unused high bits of the last word are 0.
+// STE bit masks of the re-computation pass (Sec. 4, App. D).  mask1[M][ceil(K/32)][N]: bit (i % 32) of word i / 32
+// of output (m, n) is the STE value of step i of the first hierarchy (of the only one in sequential order).
+// mask2[M][ceil(C/32)][N], C = ceil(K / chunk), chunked order only: the same for the step that folds chunk j into
+// the second hierarchy.  Unused high bits of the last word are 0.
 int lbo_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, int64_t K, const lbo_fmt* pf,
                       const lbo_fmt* af, int order, int64_t chunk, int kind, float eps1, float eps2, uint32_t* mask1,
                       uint32_t* mask2, int nthreads) {
@@ -601,10 +601,11 @@ int lbo_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, 
   if ((M * N * W1 > 0 && !mask1) || (M * N * W2 > 0 && !mask2)) return LBO_ERR_ARG;
   return parallel_items(M, nthreads, [&](int64_t m) {
     for (int64_t n = 0; n < N; ++n) {
-      uint32_t* w1 = mask1 + (m * N + n) * W1;
-      uint32_t* w2 = chunked ? mask2 + (m * N + n) * W2 : nullptr;
-      for (int64_t i = 0; i < W1; ++i) w1[i] = 0;
-      for (int64_t i = 0; i < W2; ++i) w2[i] = 0;
+      // word w of output (m, n): base[(m * words + w) * N + n]
+      auto word1 = [&](int64_t w) -> uint32_t& { return mask1[(m * W1 + w) * N + n]; };
+      auto word2 = [&](int64_t w) -> uint32_t& { return mask2[(m * W2 + w) * N + n]; };
+      for (int64_t i = 0; i < W1; ++i) word1(i) = 0;
+      for (int64_t i = 0; i < W2; ++i) word2(i) = 0;
       Chain c(&g.prod, &g.acc, g.order, g.chunk);
       c.ste_kind = kind;
       c.eps1 = eps1;
@@ -612,16 +613,16 @@ int lbo_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, 
       for (int64_t i = 0; i < K; ++i) {
         c.fmaq_step(A[m * K + i], B[n * K + i]);
         if (c.status != LBO_OK) return c.status;
-        if (c.ste_first) w1[i / 32] |= 1u << (i % 32);
+        if (c.ste_first) word1(i / 32) |= 1u << (i % 32);
         const int64_t before = c.chunks_closed;
         c.end_of_step();
         if (c.status != LBO_OK) return c.status;
-        if (c.chunks_closed != before && c.ste_second) w2[before / 32] |= 1u << (before % 32);
+        if (c.chunks_closed != before && c.ste_second) word2(before / 32) |= 1u << (before % 32);
       }
       const int64_t before = c.chunks_closed;
       c.finish();   // folds a short last chunk
       if (c.status != LBO_OK) return c.status;
-      if (c.chunks_closed != before && c.ste_second) w2[before / 32] |= 1u << (before % 32);
+      if (c.chunks_closed != before && c.ste_second) word2(before / 32) |= 1u << (before % 32);
     }
     return (int)LBO_OK;
   });

@@ -173,17 +173,17 @@ STE_OF, STE_DIFF = 1, 2
 
 
 def gemm_ste_mask(A, B, prod_fmt, acc_fmt, order, chunk, kind, eps1=0.0, eps2=0.0, nthreads=0):
-    """(mask1 uint32 [M][N][ceil(K/32)], mask2 uint32 [M][N][ceil(ceil(K/chunk)/32)] or None): STE bit of every
+    """(mask1 uint32 [M][ceil(K/32)][N], mask2 uint32 [M][ceil(ceil(K/chunk)/32)][N] or None): STE bit of every
     FMAq step of the first hierarchy and, in chunked order, of every fold into the second (App. D)."""
     A, Ap = _u8(A)
     B, Bp = _u8(B)
     M, K = A.shape
     N, _ = B.shape
     pf, af = _fmt(prod_fmt), _fmt(acc_fmt)
-    m1 = np.empty((M, N, (K + 31) // 32), dtype=np.uint32)
+    m1 = np.empty((M, (K + 31) // 32, N), dtype=np.uint32)
     m2 = None
     if order == 1:  # chunked
-        m2 = np.empty((M, N, ((K + chunk - 1) // chunk + 31) // 32), dtype=np.uint32)
+        m2 = np.empty((M, ((K + chunk - 1) // chunk + 31) // 32, N), dtype=np.uint32)
     u32 = C.POINTER(C.c_uint32)
     _check(lib().lbo_gemm_ste_mask(Ap, Bp, C.c_int64(M), C.c_int64(N), C.c_int64(K), C.byref(pf), C.byref(af),
                                    C.c_int(order), C.c_int64(chunk), C.c_int(kind), C.c_float(eps1), C.c_float(eps2),

@@ -174,17 +174,17 @@ STE_OF, STE_DIFF = 1, 2
 
 def lba_gemm_ste_mask(A, B, prod_fmt, acc_fmt, order=ORDER_CHUNKED, chunk=PAPER_CHUNK, ste=STE_OF, eps1=0.0, eps2=0.0,
                       stream=None):
-    """(mask1 int32 [M][N][ceil(K/32)], mask2 int32 [M][N][ceil(ceil(K/chunk)/32)] or None): one STE bit per FMAq
+    """(mask1 int32 [M][ceil(K/32)][N], mask2 int32 [M][ceil(ceil(K/chunk)/32)][N] or None): one STE bit per FMAq
     step, as 32-bit words (torch has no unsigned 32-bit arithmetic; the bit patterns are what counts).  See lba.h."""
     lib = load_library()
     M, K = A.shape
     N, K2 = B.shape
     if K != K2:
         raise ValueError("A and B disagree on K")
-    mask1 = torch.empty((M, N, (K + 31) // 32), dtype=torch.int32, device=A.device)
+    mask1 = torch.empty((M, (K + 31) // 32, N), dtype=torch.int32, device=A.device)
     mask2 = None
     if order == ORDER_CHUNKED:
-        mask2 = torch.empty((M, N, ((K + chunk - 1) // max(chunk, 1) + 31) // 32), dtype=torch.int32, device=A.device)
+        mask2 = torch.empty((M, ((K + chunk - 1) // max(chunk, 1) + 31) // 32, N), dtype=torch.int32, device=A.device)
     pf, af = _fmt(prod_fmt), _fmt(acc_fmt)
     _check(lib.lba_gemm_ste_mask(_dev(A, torch.uint8, "A"), _dev(B, torch.uint8, "B"), M, N, K, C.byref(pf), C.byref(af),
                                  order, chunk, ste, C.c_float(eps1), C.c_float(eps2), _dev(mask1, torch.int32, "mask1"),

@@ -315,8 +315,8 @@ struct RowLoader {
 //   TRACK_MASK_OF  one bit per FMAq step, 1 iff |Q_prod(x_i w_i) + S_i| < R_OF (STE^OF);
 //   TRACK_MASK_DIFF one bit per FMAq step, 1 iff |z - S| > eps2 * (|x_i w_i| + eps1) (STE^DIFF), each of the three
 //                  operations rounded to binary32.
-// Masks: mask1 uint32 [M][N][ceil(K/32)], bit i%32 of word i/32 for step i; in chunked order mask2
-// [M][N][ceil(chunks/32)] holds the bits of the folds T <- Q_acc(C + T), the chunk sum C in the product's place.
+// Masks: mask1 uint32 [M][ceil(K/32)][N], bit i%32 of word i/32 for step i; in chunked order mask2
+// [M][ceil(chunks/32)][N] holds the bits of the folds T <- Q_acc(C + T), the chunk sum C in the product's place.
 enum { TRACK_NONE = 0, TRACK_LAST_OF = 1, TRACK_MASK_OF = 2, TRACK_MASK_DIFF = 3 };
 
 template <int BM, int BN, int TM, int TN, int QM, int ORD, int LD, int TRACK = TRACK_NONE>
@@ -406,16 +406,28 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
   const int64_t W2 = MASKS ? p.mask2_words : 0;
   const float dscale = p.diff_scale, deps1 = p.diff_eps1, deps2 = p.diff_eps2;
 
-  // one word of a mask for every output of the thread
+  // one word of a mask for every output of the thread: word w of output (m, n) is base[(m * words + w) * N + n],
+  // so the four neighbouring outputs of a micro-tile row go out as one 16-byte store where alignment allows
   auto flush_words = [&](uint32_t* base, int64_t words, int64_t w, auto& bits) {
+    const bool vec = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(base) & 15) == 0);
 #pragma unroll
     for (int i = 0; i < TM; ++i) {
       const int64_t m = m0 + (i / 4) * (BM / 2) + ty * 4 + (i % 4);
 #pragma unroll
-      for (int j = 0; j < TN; ++j) {
-        const int64_t n = n0 + (j / 4) * (BN / 2) + tx * 4 + (j % 4);
-        if (m < p.M && n < p.N) base[(m * p.N + n) * words + w] = bits[i][j];
-        bits[i][j] = 0u;
+      for (int h = 0; h < TN / 4; ++h) {
+        const int64_t n = n0 + h * (BN / 2) + tx * 4;
+        uint32_t* dst = base + (m * words + w) * p.N + n;
+        if (m < p.M) {
+          if (vec && n + 3 < p.N) {
+            *reinterpret_cast<uint4*>(dst) = make_uint4(bits[i][h * 4], bits[i][h * 4 + 1], bits[i][h * 4 + 2], bits[i][h * 4 + 3]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              if (n + j < p.N) dst[j] = bits[i][h * 4 + j];
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) bits[i][h * 4 + j] = 0u;
       }
     }
   };

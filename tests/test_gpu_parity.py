@@ -374,11 +374,11 @@ def test_ste_mask_edge_cases():
     a = torch.full((1, 300), 0x30, dtype=torch.uint8, device=DEV)
     w = torch.full((1, 300), 0x28, dtype=torch.uint8, device=DEV)
     m1, _ = lba.lba_gemm_ste_mask(a, w, prod, acc, SEQ, 1, lba.STE_DIFF, 1e-6, 0.5)
-    assert [int(v) & 0xFFFFFFFF for v in m1[0, 0]] == [0xFFFFFFFF] * 8 + [0, 0]
+    assert [int(v) & 0xFFFFFFFF for v in m1[0, :, 0]] == [0xFFFFFFFF] * 8 + [0, 0]
     # empty problems, K = 0
     e1, e2 = lba.lba_gemm_ste_mask(torch.empty((3, 0), dtype=torch.uint8, device=DEV),
                                    torch.empty((2, 0), dtype=torch.uint8, device=DEV), prod, acc, CHK, 16, lba.STE_OF)
-    assert e1.shape == (3, 2, 0) and e2.shape == (3, 2, 0)
+    assert e1.shape == (3, 0, 2) and e2.shape == (3, 0, 2)
     # odd base pointers: byte-wise loader
     Abig = (synth.random_codes((40 * 64 + 3,), 3) & 0x7F).to(DEV)
     Bbig = (synth.random_codes((33 * 64 + 5,), 4) & 0x7F).to(DEV)

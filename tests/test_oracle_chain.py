@@ -249,20 +249,20 @@ def test_ste_masks_hand_worked_chains():
     a = np.full((1, 300), 0x30, np.uint8)
     w = np.full((1, 300), 0x28, np.uint8)
     m1, _ = orc.gemm_ste_mask(a, w, prod, acc, 0, 1, orc.STE_DIFF, 1e-6, 0.5)
-    assert _bits_of(m1[0, 0], 300) == [1] * 256 + [0] * 44
-    assert (m1[0, 0, 9] >> 12) == 0                                   # unused high bits of the last word
+    assert m1.shape == (1, 10, 1) and _bits_of(m1[0, :, 0], 300) == [1] * 256 + [0] * 44
+    assert (m1[0, 9, 0] >> 12) == 0                                   # unused high bits of the last word
     m1, _ = orc.gemm_ste_mask(a, w, prod, acc, 0, 1, orc.STE_OF)
-    assert _bits_of(m1[0, 0], 300) == [1] * 300
+    assert _bits_of(m1[0, :, 0], 300) == [1] * 300
     # chunks of 16 keep every first-level sum at <= 2.0 and the folds add 2.0 to T <= 37.5 exactly: all bits pass
     m1, m2 = orc.gemm_ste_mask(a, w, prod, acc, 1, 16, orc.STE_DIFF, 1e-6, 0.5)
-    assert _bits_of(m1[0, 0], 300) == [1] * 300 and _bits_of(m2[0, 0], 19) == [1] * 19 and m2.shape == (1, 1, 1)
+    assert _bits_of(m1[0, :, 0], 300) == [1] * 300 and _bits_of(m2[0, :, 0], 19) == [1] * 19 and m2.shape == (1, 1, 1)
     # K = 576 in chunks of 16: T climbs by 2.0 per fold and saturates at 63.75 at the 32nd fold (exact sum 64):
     # STE^OF of the folds is 1 for folds 0..30 and 0 from fold 31 on
     a = np.full((1, 576), 0x30, np.uint8)
     w = np.full((1, 576), 0x28, np.uint8)
     m1, m2 = orc.gemm_ste_mask(a, w, prod, acc, 1, 16, orc.STE_OF)
-    assert _bits_of(m2[0, 0], 36) == [1] * 31 + [0] * 5 and m2.shape == (1, 1, 2)
-    assert all(v == 0xFFFFFFFF for v in m1[0, 0])
+    assert _bits_of(m2[0, :, 0], 36) == [1] * 31 + [0] * 5 and m2.shape == (1, 2, 1)
+    assert all(v == 0xFFFFFFFF for v in m1[0, :, 0])
     # a single chunk still has its fold: x = w = 4.0, K = 7, chunk 16: C = 63.75 (saturated), |C + 0| >= R_OF
     x = np.full((1, 7), 0x48, np.uint8)
     m1, m2 = orc.gemm_ste_mask(x, x, prod, acc, 1, 16, orc.STE_OF)
@@ -293,8 +293,8 @@ def test_ste_masks_against_exact_rationals_and_last_overflow():
             for m in range(2):
                 for n in range(2):
                     f, s = ex.ste_bits(pf, af, order, chunk, A[m], B[n], name, e1, e2)
-                    assert _bits_of(m1[m, n], K) == f
-                    assert order == 0 or _bits_of(m2[m, n], len(s)) == s
+                    assert _bits_of(m1[m, :, n], K) == f
+                    assert order == 0 or _bits_of(m2[m, :, n], len(s)) == s
                     zeros += f.count(0)
                     ones += f.count(1)
                     if kind == orc.STE_OF and order == 0:
