@@ -32,6 +32,8 @@ BATCH = 32
 CONFIG_ID = 2
 RUN_ORDER = 1        # ORDER_CHUNKED, the paper's order; a single-GEMM workload may ask for the sequential order
 GEMM_CASE = None     # (M, N, K) when --workload gemm:MxNxK[:seq|chunk] replaces the network
+STE_KIND = None      # "of" / "diff" when --workload ste:... times the mask re-computation pass
+STE_EPS = (2.0 ** -20, 0.25)
 
 # ALU roofline for sm_100.  Per SM and clock 4 schedulers issue one warp instruction each (128 lanes), the
 # FP32 pipe retires 128 lanes and the integer/logic pipe 64.  The packed floor path needs, per emulated MAC,
@@ -69,7 +71,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet18",
                     help="resnet18 (default, the benchmark), gemm:MxNxK[:seq|chunk] (one LBA GEMM on Gaussian "
-                         "operands, used for kernel profiles) or bgemm:ZxMxNxK[:seq|chunk] (one batched call)")
+                         "operands, used for kernel profiles), bgemm:ZxMxNxK[:seq|chunk] (one batched call) or "
+                         "ste:MxNxK[:of|diff][:seq|chunk] (STE mask re-computation of one GEMM)")
     ap.add_argument("--cpu-baseline-macs", type=float, default=1.5e9,
                     help="size of the oracle sample timed for cpu_baseline (emulated MACs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -164,6 +167,10 @@ def build_calls(device):
         a, sa, b, sb = synth.gemm_case(m, n, k, config=5)
         c = workloads.LbaCall("gemm", "gemm", a.to(device), b.to(device), sa.to(device), sb.to(device))
         c.out = torch.empty((m, n), dtype=torch.float32, device=device)
+        if STE_KIND is not None:
+            c.kind = "ste"
+            c.mask1 = torch.empty((m, (k + 31) // 32, n), dtype=torch.int32, device=device)
+            c.mask2 = torch.empty((m, ((k + 15) // 16 + 31) // 32, n), dtype=torch.int32, device=device) if RUN_ORDER else None
         return [c]
 
     def conv_fn(x, w, sx, sw, stride, pad):
@@ -190,6 +197,9 @@ def run_step(calls, events=None):
             lba.lba_conv2d(c.x, c.w, c.sx, c.sw, None, c.stride, c.pad, prod, acc, ORDER_CHUNKED, 16, out=c.out_nhwc)
         elif c.kind == "bgemm":
             lba.lba_gemm_batched(c.x, c.w, c.sx, c.sw, None, prod, acc, ORDER_CHUNKED, 16, out=c.out)
+        elif c.kind == "ste":
+            lba.lba_gemm_ste_mask(c.x, c.w, prod, acc, ORDER_CHUNKED, 16, lba.STE_DIFF if STE_KIND == "diff" else lba.STE_OF,
+                                  STE_EPS[0], STE_EPS[1], mask1=c.mask1, mask2=c.mask2)
         else:
             lba.lba_gemm(c.x, c.w, c.sx, c.sw, None, prod, acc, ORDER_CHUNKED, 16, out=c.out)
         if events is not None:
@@ -201,6 +211,8 @@ def describe(c):
     ORDER_CHUNKED = RUN_ORDER
     prod, acc = formats()
     m, n, k = c.gemm_shape
+    if c.kind == "ste":
+        return "ste_mask=%s tile=64x64x16 micro=4x4 q=floor order=%s" % (STE_KIND, "chunk16" if RUN_ORDER else "seq")
     vec = (c.x.shape[-1] % 16 == 0) if c.kind == "conv" else (k % 16 == 0)
     return lba.describe_plan(m, n, k, prod, acc, ORDER_CHUNKED, 16, is_conv=c.kind == "conv", vec_ok=vec)
 
@@ -283,7 +295,7 @@ def reference_arm(args):
 
 
 def main():
-    global WORKLOAD, RUN_ORDER, GEMM_CASE
+    global WORKLOAD, RUN_ORDER, GEMM_CASE, STE_KIND
     args = parse_args()
     if args.workload.startswith("bgemm:"):
         parts = args.workload.split(":")
@@ -298,6 +310,14 @@ def main():
         GEMM_CASE = tuple(int(v) for v in parts[1].lower().split("x"))
         RUN_ORDER = 0 if (len(parts) > 2 and parts[2].startswith("seq")) else 1
         WORKLOAD = "single_lba_gemm_%dx%dx%d_m7e4_%s" % (GEMM_CASE + ("sequential" if RUN_ORDER == 0 else "chunk16",))
+    elif args.workload.startswith("ste:"):
+        # ste:MxNxK[:of|diff][:seq|chunk]: the mask re-computation pass of the straight-through estimators
+        parts = args.workload.split(":")
+        GEMM_CASE = tuple(int(v) for v in parts[1].lower().split("x"))
+        STE_KIND = "diff" if "diff" in parts[2:] else "of"
+        RUN_ORDER = 0 if "seq" in parts[2:] else 1
+        WORKLOAD = "ste_%s_mask_%dx%dx%d_m7e4_%s" % ((STE_KIND,) + GEMM_CASE + ("sequential" if RUN_ORDER == 0 else "chunk16",))
+        args.no_e2e = args.no_cpu_baseline = True      # kernel timing only for this workload
     elif args.workload != "resnet18":
         raise SystemExit("unknown --workload")
     if args.impl == "reference":
@@ -373,6 +393,13 @@ def main():
     max_mhz = clocks["sm_max_mhz"] or 1965.0
     mhz = clocks["sm_mhz"] or max_mhz
     slots = issue_slots_per_mac(RUN_ORDER == 1, 16)
+    mix = "0.5 FMUL2 + 0.5 FFMA2 + 1 LOP3, plus 2.5 per output per chunk of 16"
+    if STE_KIND is not None:
+        # scalar tracking kernel: multiply, add (toward zero), mantissa mask, compare with R_OF, clamp, bit insert;
+        # the difference estimator adds the rescaled sum, the subtraction, |x w|, + eps1, * eps2
+        slots = (6.0 if STE_KIND == "of" else 11.0) + (slots - ISSUE_SLOTS_PER_MAC_LEVEL1)
+        mix = ("FMUL + FFMA + LOP3 + FSETP + FMNMX + bit insert" if STE_KIND == "of" else
+               "FMUL + FFMA + LOP3 + FMNMX + 3 FMUL + 2 FADD + FSETP + bit insert") + ", scalar, plus the chunk folds"
     peak = sm_count * ISSUE_LANES_PER_SM_CLK * max_mhz * 1e6 / slots / 1e9
     achieved = dom["macs"] / (dom["ms"] * 1e-3) / 1e9
     roofline = {
@@ -382,11 +409,15 @@ def main():
         "kernel": dom_key, "kernel_launches_per_step": dom["launches"], "kernel_ms_per_step": dom["ms"],
         "kernel_share_of_step": dom["ms"] / sum(per_call_ms),
         "peak_derivation": f"{sm_count} SMs x {ISSUE_LANES_PER_SM_CLK} lanes issued per clock x {max_mhz:.0f} MHz "
-                           f"(clocks.max.sm) / {slots:g} issue slots per emulated MAC (0.5 FMUL2 + 0.5 FFMA2 + 1 LOP3, "
-                           f"plus 2.5 per output per chunk of 16); the FP32 and logic pipes give the same limit",
+                           f"(clocks.max.sm) / {slots:g} issue slots per emulated MAC ({mix})"
+                           + ("; the FP32 and logic pipes give the same limit" if STE_KIND is None else ""),
         "frac_at_sampled_clock": achieved / (peak * mhz / max_mhz),
         "whole_step_frac_of_peak": (step_macs / (sum(per_call_ms) * 1e-3) / 1e9) / peak,
     }
+    if STE_KIND is not None:   # one bit per step: the masks are the bulk of the algorithmic bytes
+        mask_bytes = sum(c.mask1.numel() * 4 + (c.mask2.numel() * 4 if c.mask2 is not None else 0) for c in calls)
+        roofline["mask_bytes_per_launch"] = mask_bytes
+        roofline["mask_write_gbs"] = mask_bytes / (dom["ms"] * 1e-3) / 1e9
 
     # ---- end to end through the host-buffer C entry points
     e2e = None

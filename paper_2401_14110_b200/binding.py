@@ -173,7 +173,7 @@ STE_OF, STE_DIFF = 1, 2
 
 
 def lba_gemm_ste_mask(A, B, prod_fmt, acc_fmt, order=ORDER_CHUNKED, chunk=PAPER_CHUNK, ste=STE_OF, eps1=0.0, eps2=0.0,
-                      stream=None):
+                      mask1=None, mask2=None, stream=None):
     """(mask1 int32 [M][ceil(K/32)][N], mask2 int32 [M][ceil(ceil(K/chunk)/32)][N] or None): one STE bit per FMAq
     step, as 32-bit words (torch has no unsigned 32-bit arithmetic; the bit patterns are what counts).  See lba.h."""
     lib = load_library()
@@ -181,9 +181,11 @@ def lba_gemm_ste_mask(A, B, prod_fmt, acc_fmt, order=ORDER_CHUNKED, chunk=PAPER_
     N, K2 = B.shape
     if K != K2:
         raise ValueError("A and B disagree on K")
-    mask1 = torch.empty((M, (K + 31) // 32, N), dtype=torch.int32, device=A.device)
-    mask2 = None
-    if order == ORDER_CHUNKED:
+    if mask1 is None:
+        mask1 = torch.empty((M, (K + 31) // 32, N), dtype=torch.int32, device=A.device)
+    if order != ORDER_CHUNKED:
+        mask2 = None
+    elif mask2 is None:
         mask2 = torch.empty((M, ((K + chunk - 1) // max(chunk, 1) + 31) // 32, N), dtype=torch.int32, device=A.device)
     pf, af = _fmt(prod_fmt), _fmt(acc_fmt)
     _check(lib.lba_gemm_ste_mask(_dev(A, torch.uint8, "A"), _dev(B, torch.uint8, "B"), M, N, K, C.byref(pf), C.byref(af),

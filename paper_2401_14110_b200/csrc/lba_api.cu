@@ -22,8 +22,8 @@ LBA_DECL(QM_RNE_WIDE, ORD_SEQ) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_SLAB) LBA_DECL(QM
 
 cudaError_t launch_umma_family(int load, const Problem& p, cudaStream_t stream);
 cudaError_t read_umma_error(int* code);
-cudaError_t launch_last_overflow(int load, const Problem& p, cudaStream_t stream);
-cudaError_t launch_ste_mask(int ord, int diff, int load, const Problem& p, cudaStream_t stream);
+cudaError_t launch_last_overflow(int qm, int load, const Problem& p, cudaStream_t stream);
+cudaError_t launch_ste_mask(int qm, int ord, int diff, int load, const Problem& p, cudaStream_t stream);
 
 namespace {
 
@@ -440,7 +440,7 @@ int lba_gemm_last_overflow(const uint8_t* A, const uint8_t* B, int64_t M, int64_
   p.out = reinterpret_cast<float*>(last);
   apply_plan(&p, pl);
   const bool vec = K % BK == 0 && aligned16(A) && aligned16(B);
-  const cudaError_t e = launch_last_overflow(vec ? LD_GEMM_VEC : LD_ANY, p, (cudaStream_t)stream);
+  const cudaError_t e = launch_last_overflow(pl.qm, vec ? LD_GEMM_VEC : LD_ANY, p, (cudaStream_t)stream);
   return e == cudaSuccess ? LBA_OK : cuda_fail(e);
 }
 
@@ -505,7 +505,7 @@ int lba_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, 
     p.chunk_slabs = chunk / BK;
   }
   const bool vec = K % BK == 0 && aligned16(A) && aligned16(B);
-  const cudaError_t e = launch_ste_mask(ord, ste == LBA_STE_DIFF, vec ? LD_GEMM_VEC : LD_ANY, p, (cudaStream_t)stream);
+  const cudaError_t e = launch_ste_mask(pl.qm, ord, ste == LBA_STE_DIFF, vec ? LD_GEMM_VEC : LD_ANY, p, (cudaStream_t)stream);
   return e == cudaSuccess ? LBA_OK : cuda_fail(e);
 }
 

@@ -321,7 +321,7 @@ enum { TRACK_NONE = 0, TRACK_LAST_OF = 1, TRACK_MASK_OF = 2, TRACK_MASK_DIFF = 3
 
 template <int BM, int BN, int TM, int TN, int QM, int ORD, int LD, int TRACK = TRACK_NONE>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(const Problem p) {
-  static_assert(TRACK == TRACK_NONE || QM == QM_FLOOR_FULL, "tracking variants use the floor quantisers");
+  static_assert(TRACK == TRACK_NONE || QM == QM_FLOOR_FULL || QM == QM_FLOOR_FAST, "tracking variants use the floor quantisers");
   static_assert(TRACK != TRACK_LAST_OF || ORD == ORD_SEQ, "last-overflow index: sequential order");
   static_assert(TRACK == TRACK_NONE || ORD != ORD_CHUNK16, "tracking variants: generic orders");
   constexpr bool MASKS = TRACK == TRACK_MASK_OF || TRACK == TRACK_MASK_DIFF;
@@ -385,6 +385,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
   constexpr bool LAST = TRACK == TRACK_LAST_OF;
   int last[LAST ? TM : 1][LAST ? TN : 1];                       // TRACK_LAST_OF
   uint32_t bits1[MASKS ? TM : 1][MASKS ? TN : 1];               // current word of mask1
+  uint32_t half1[MASKS ? TM : 1][MASKS ? TN : 1];               // the 16 bits of the current slab
   uint32_t bits2[MASKS && CHUNKED ? TM : 1][MASKS && CHUNKED ? TN : 1];
   float prev1[DIFF ? TM : 1][DIFF ? TN : 1];                    // S and T in the comparison's scaling
   float prev2[DIFF && CHUNKED ? TM : 1][DIFF && CHUNKED ? TN : 1];
@@ -393,7 +394,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
 #pragma unroll
     for (int j = 0; j < TN; ++j) {
       if (LAST) last[LAST ? i : 0][LAST ? j : 0] = -1;
-      if (MASKS) bits1[MASKS ? i : 0][MASKS ? j : 0] = 0u;
+      if (MASKS) bits1[MASKS ? i : 0][MASKS ? j : 0] = half1[MASKS ? i : 0][MASKS ? j : 0] = 0u;
       if (MASKS && CHUNKED) bits2[MASKS && CHUNKED ? i : 0][MASKS && CHUNKED ? j : 0] = 0u;
       if (DIFF) prev1[DIFF ? i : 0][DIFF ? j : 0] = 0.0f;
       if (DIFF && CHUNKED) prev2[DIFF && CHUNKED ? i : 0][DIFF && CHUNKED ? j : 0] = 0.0f;
@@ -434,16 +435,16 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
 
   // STE bit of one step: t = the exact sum cut toward zero to M bits (|t| >= R_OF exactly when the exact
   // sum is), z = Q_acc of it, u = the unquantised product or the chunk sum (DIFF scaling), s_prev = S before
-  auto ste_bit = [&](float t, float z, float u, float& s_prev) -> uint32_t {
+  auto ste_bit = [&](float t, float z, float u, float& s_prev) -> bool {
     if (DIFF) {
       const float zd = mul_ieee(z, dscale);                       // exact: z is a normal number
       const float d = fabsf(__fadd_rn(zd, -s_prev));              // one rounding, as the definition says
       s_prev = zd;
       const float thr = __fmul_rn(deps2, __fadd_rn(fabsf(u), deps1));
-      return d > thr ? 1u : 0u;
+      return d > thr;
     }
     (void)z; (void)u; (void)s_prev;
-    return fabsf(t) < qa.sat ? 1u : 0u;
+    return fabsf(t) < qa.sat;
   };
 
   auto close_chunk = [&]() {  // second hierarchy: T <- Q_acc(C + T), C <- 0
@@ -456,8 +457,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
           const float t = and_bits(fma_rz_ftz(acc1[i][j], 1.0f, t2), qa.mask);
           const float z = clamp_mag(t, qa.sat);
           const float u = DIFF ? mul_ieee(acc1[i][j], dscale) : 0.0f;
-          bits2[MASKS && CHUNKED ? i : 0][MASKS && CHUNKED ? j : 0] |=
-              ste_bit(t, z, u, prev2[DIFF && CHUNKED ? i : 0][DIFF && CHUNKED ? j : 0]) << (chunk_id & 31);
+          if (ste_bit(t, z, u, prev2[DIFF && CHUNKED ? i : 0][DIFF && CHUNKED ? j : 0]))
+            bits2[MASKS && CHUNKED ? i : 0][MASKS && CHUNKED ? j : 0] |= 1u << (chunk_id & 31);
           t2 = z;
           if (DIFF) prev1[DIFF ? i : 0][DIFF ? j : 0] = 0.0f;
         } else {
@@ -502,8 +503,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
             if (fabsf(t) >= qa.sat && real_step) last[LAST ? i : 0][LAST ? j : 0] = kbase + kk;
           } else {
             const float u = DIFF ? mul_ieee(ad[DIFF ? i : 0], b[j]) : 0.0f;  // exact |x w| in the comparison's scaling
-            const uint32_t bit = ste_bit(t, z, u, prev1[DIFF ? i : 0][DIFF ? j : 0]);
-            bits1[MASKS ? i : 0][MASKS ? j : 0] |= (real_step ? bit : 0u) << ((kbase + kk) & 31);
+            // bit kk of the slab's halfword; steps past K are cleared when the halfword joins its word
+            if (ste_bit(t, z, u, prev1[DIFF ? i : 0][DIFF ? j : 0])) half1[MASKS ? i : 0][MASKS ? j : 0] |= 1u << kk;
           }
           acc1[i][j] = z;
         } else {
@@ -544,7 +545,17 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(con
         }
       }
     }
-    if constexpr (MASKS) {  // a word of mask1 is complete after every second slab
+    if constexpr (MASKS) {  // the slab's 16 bits join their word; a word is complete after every second slab
+      const int valid = (int)((K - kbase) < BK ? (K - kbase) : BK);
+      const uint32_t keep = valid >= 16 ? 0xFFFFu : ((1u << valid) - 1u);
+      const int sh = (s & 1) * 16;
+#pragma unroll
+      for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) {
+          bits1[i][j] |= (half1[i][j] & keep) << sh;
+          half1[i][j] = 0u;
+        }
       if ((s & 1) || s + 1 == nslab) flush_words(mask1z, W1, (int64_t)(s >> 1), bits1);
     }
     if (s + 1 < nslab) decode_store(raw, buf ^ 1);

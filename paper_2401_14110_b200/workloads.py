@@ -99,7 +99,7 @@ class LbaCall:
     def gemm_shape(self):
         if self.kind == "bgemm":        # per problem; macs counts all of them
             return self.x.shape[1], self.w.shape[1], self.x.shape[2]
-        if self.kind == "gemm":
+        if self.kind in ("gemm", "ste"):   # "ste": the mask re-computation pass of the same GEMM
             return self.x.shape[0], self.w.shape[0], self.x.shape[1]
         b, h, wd, cin = self.x.shape
         cout, kh, kw, _ = self.w.shape
