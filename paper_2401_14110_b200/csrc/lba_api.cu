@@ -210,7 +210,7 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
 // Tile choice.  All CTAs of a launch have the same work and K is never split, so the launch ends when the
 // busiest SM has run its ceil(CTAs / SMs) tiles; larger tiles spend fewer instructions per MAC (eff, measured
 // on B200 with every SM loaded), smaller ones fill the SMs more evenly.  Pick the cheapest by that model.
-int choose_tile(int64_t M, int64_t N, int64_t batch, int qm, int ord) {
+int choose_tile(int64_t M, int64_t N, int64_t batch, int qm, int ord, int load) {
   (void)qm;
   if (g_tile_override >= 0 && g_tile_override < TILE_COUNT) return g_tile_override;
   int dev = 0, sms = 148;
@@ -221,7 +221,10 @@ int choose_tile(int64_t M, int64_t N, int64_t batch, int qm, int ord) {
   // relative MAC rate of each tile with every SM loaded (8192^2 x 1024 and 4096 x 3072 x 768 GEMMs)
   const double eff_seq[TILE_COUNT] = {1.00, 0.91, 0.95, 0.84};
   const double eff_chunk[TILE_COUNT] = {0.97, 0.96, 1.00, 0.89};
-  const double* eff = ord == ORD_SEQ ? eff_seq : eff_chunk;
+  // byte-wise loader (ResNet stem, 401408 x 64 x 147): the fetch is costly, so the tile with the fewest
+  // fetched rows per output wins as long as it keeps its registers
+  const double eff_any[TILE_COUNT] = {0.55, 1.00, 0.87, 0.73};
+  const double* eff = load == LD_ANY ? eff_any : (ord == ORD_SEQ ? eff_seq : eff_chunk);
   int best = 0;
   double best_cost = 1e300;
   for (int t = 0; t < TILE_COUNT; ++t) {
@@ -282,7 +285,7 @@ int run(const Problem& p, const Plan& pl, int load, cudaStream_t stream) {
       return e == cudaSuccess ? LBA_OK : cuda_fail(e);
     }
   }
-  const int tile = choose_tile(p.M, p.N, p.batch, pl.qm, pl.ord);
+  const int tile = choose_tile(p.M, p.N, p.batch, pl.qm, pl.ord, load);
   const TileInfo ti = tile_info(tile);
   if ((p.N + ti.bn - 1) / ti.bn > 65535 || (p.M + ti.bm - 1) / ti.bm > 2147483647LL) return LBA_ERR_SHAPE;
   const cudaError_t e = kLaunch[pl.qm][pl.ord](tile, load, p, stream);
@@ -651,9 +654,9 @@ int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, 
   Plan pl;
   const int st = make_plan(prod_fmt, acc_fmt, order, chunk, K, &pl);
   if (st != LBA_OK) return st;
-  const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, 1, pl.qm, pl.ord);
-  const TileInfo ti = tile_info(tile);
   const int load = vec_ok ? (is_conv ? LD_CONV_VEC : LD_GEMM_VEC) : LD_ANY;
+  const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, 1, pl.qm, pl.ord, load);
+  const TileInfo ti = tile_info(tile);
   if (buf && buf_len)
     std::snprintf(buf, buf_len, "tile=%dx%dx%d micro=%dx%d q=%s order=%s load=%s grid=%lldx%lld", ti.bm, ti.bn, BK,
                   ti.tm, ti.tn, kQmName[pl.qm], kOrdName[pl.ord], kLdName[load], (long long)((M + ti.bm - 1) / ti.bm),

@@ -772,7 +772,8 @@ __host__ __device__ constexpr int packed_tmem_cols() {
 }
 
 // the 8x8 micro-tile is held to 128 registers (two CTAs of 256 threads per SM) wherever the second-level
-// sums are not in registers
+// sums are not in registers; so is the byte-wise loader, whose sixteen loads in flight would otherwise
+// cost fifty registers and half the resident CTAs
 // PQ: what Q_prod has to do beyond the flush (the host proves which cases are reachable): nothing, cut the
 // mantissa (M_prod < 7), or cut and saturate (448^2 >= R_OF_prod)
 enum PackedProd { PQ_NONE = 0, PQ_MASK = 1, PQ_MASK_SAT = 2 };
@@ -781,7 +782,8 @@ enum PackedProd { PQ_NONE = 0, PQ_MASK = 1, PQ_MASK_SAT = 2 };
 // can raise a magnitude, so the slab-level proof that the clamp is idle is not used: it always clamps.
 template <int BM, int BN, int TM, int TN, int PQ, bool RNE, int ORD, int LD>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN),
-                                  (TM * TN == 64 && ORD != ORD_CHUNK_SLAB && !RNE) ? 512 / ((BM / TM) * (BN / TN)) : 1)
+                                  ((TM * TN == 64 && ORD != ORD_CHUNK_SLAB && !RNE) || (LD == LD_ANY && !RNE && ORD != ORD_CHUNK_SLAB))
+                                      ? 512 / ((BM / TM) * (BN / TN)) : 1)
     lba_contract_packed_kernel(const Problem p) {
   constexpr int NT = (BM / TM) * (BN / TN);
   constexpr int TX = BN / TN;
