@@ -77,6 +77,8 @@ def parse_args():
                     help="size of the oracle sample timed for cpu_baseline (emulated MACs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-streams", type=int, default=12,
+                    help="streams (each with its own device workspace) the end-to-end calls are spread over")
     ap.add_argument("--force-dist", action="store_true",
                     help="initialise torch.distributed (NCCL) even for a single rank: exercises the multi-GPU plumbing "
                          "(barrier, max over ranks) on one GPU")
@@ -440,8 +442,8 @@ def main():
             d2h += 4 * hout.numel()
             host.append((c, hx, hw_, hsx, hsw, hout))
         # the calls of a step are independent here (operands recorded beforehand), so they are spread round-robin
-        # over three streams, each with its own workspace: one call's copies overlap another call's kernel
-        n_streams = 3
+        # over a few streams, each with its own workspace: one call's copies overlap another call's kernel
+        n_streams = max(1, args.e2e_streams)
         streams = [torch.cuda.Stream(device=device) for _ in range(n_streams)]
         wss = [torch.empty(ws_bytes, dtype=torch.uint8, device=device) for _ in range(n_streams)]
         torch.cuda.synchronize()
@@ -466,7 +468,7 @@ def main():
         e2e = {"value": sharding.whole_job_rate(step_macs, world, e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
                "api": "lba_conv2d_host / lba_gemm_host (pinned host buffers, caller-owned device workspaces, "
-                      "3 streams round-robin)"}
+                      f"{n_streams} streams round-robin)"}
         del wss, host
 
     cpu = None
