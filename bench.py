@@ -188,22 +188,24 @@ def build_calls(device):
     return calls
 
 
-def run_step(calls, events=None):
+def run_step(calls, events=None, streams=None):
     from paper_2401_14110_b200 import binding as lba
     ORDER_CHUNKED = RUN_ORDER
     prod, acc = formats()
     for i, c in enumerate(calls):
         if events is not None:
             events[i][0].record()
+        st = None if streams is None else streams[i % len(streams)]
         if c.kind == "conv":
-            lba.lba_conv2d(c.x, c.w, c.sx, c.sw, None, c.stride, c.pad, prod, acc, ORDER_CHUNKED, 16, out=c.out_nhwc)
+            lba.lba_conv2d(c.x, c.w, c.sx, c.sw, None, c.stride, c.pad, prod, acc, ORDER_CHUNKED, 16, out=c.out_nhwc,
+                           stream=st)
         elif c.kind == "bgemm":
             lba.lba_gemm_batched(c.x, c.w, c.sx, c.sw, None, prod, acc, ORDER_CHUNKED, 16, out=c.out)
         elif c.kind == "ste":
             lba.lba_gemm_ste_mask(c.x, c.w, prod, acc, ORDER_CHUNKED, 16, lba.STE_DIFF if STE_KIND == "diff" else lba.STE_OF,
                                   STE_EPS[0], STE_EPS[1], mask1=c.mask1, mask2=c.mask2)
         else:
-            lba.lba_gemm(c.x, c.w, c.sx, c.sw, None, prod, acc, ORDER_CHUNKED, 16, out=c.out)
+            lba.lba_gemm(c.x, c.w, c.sx, c.sw, None, prod, acc, ORDER_CHUNKED, 16, out=c.out, stream=st)
         if events is not None:
             events[i][1].record()
 
@@ -421,6 +423,29 @@ def main():
         roofline["mask_bytes_per_launch"] = mask_bytes
         roofline["mask_write_gbs"] = mask_bytes / (dom["ms"] * 1e-3) / 1e9
 
+    # ---- the same device-resident step with its (independent) calls spread over several streams: kernels of
+    # different calls share the SMs, which fills the tail waves a serial sequence leaves idle.  Reported beside
+    # `value`, which stays the serial figure a layer-by-layer forward pass would see.
+    concurrent = None
+    if GEMM_CASE is None and args.e2e_streams > 1:
+        cstreams = [torch.cuda.Stream(device=device) for _ in range(args.e2e_streams)]
+        barrier()
+        run_step(calls, streams=cstreams)
+        barrier()
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        for st in cstreams:
+            st.wait_event(c0)
+        for _ in range(args.steps):
+            run_step(calls, streams=cstreams)
+        for st in cstreams:
+            torch.cuda.current_stream().wait_stream(st)
+        c1.record()
+        barrier()
+        cms = sharding.max_over_ranks(c0.elapsed_time(c1), dist, device) / args.steps
+        concurrent = {"value": sharding.whole_job_rate(step_macs, world, cms * 1e-3) / 1e9, "unit": UNIT,
+                      "ms_per_step": cms, "streams": args.e2e_streams}
+
     # ---- end to end through the host-buffer C entry points
     e2e = None
     if not args.no_e2e:
@@ -489,7 +514,7 @@ def main():
                              f"outputs, larger than the 126 MB L2",
                        "parallelism": f"dp{world} (batch sharded, weights replicated, no collective)"},
             "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
+            "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "concurrent": concurrent,
             "kernels": {k: {"ms_per_step": v["ms"], "launches_per_step": v["launches"],
                             "gmacs": v["macs"] / (v["ms"] * 1e-3) / 1e9} for k, v in by_kernel.items()},
         }

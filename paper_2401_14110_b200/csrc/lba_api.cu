@@ -24,6 +24,7 @@ cudaError_t launch_umma_family(int load, const Problem& p, cudaStream_t stream);
 cudaError_t read_umma_error(int* code);
 cudaError_t launch_last_overflow(int qm, int load, const Problem& p, cudaStream_t stream);
 cudaError_t launch_ste_mask(int qm, int ord, int diff, int load, const Problem& p, cudaStream_t stream);
+cudaError_t launch_ste_packed(int pq, int chunk16, int load, const Problem& p, cudaStream_t stream);
 
 namespace {
 
@@ -500,6 +501,7 @@ int lba_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, 
   p.mask1 = mask1;
   p.mask2 = mask2;
   p.mask2_words = (chunks + 31) / 32;
+  p.ste_limit = (float)(0.999 * (1.0 - std::ldexp(1.0, -(acc_fmt->man_bits + 1))));
   // the single-chunk shortcut of the forward pass does not apply: the fold of that one chunk is a step too
   int ord = ORD_SEQ;
   if (chunked) {
@@ -508,7 +510,12 @@ int lba_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, 
     p.chunk_slabs = chunk / BK;
   }
   const bool vec = K % BK == 0 && aligned16(A) && aligned16(B);
-  const cudaError_t e = launch_ste_mask(pl.qm, ord, ste == LBA_STE_DIFF, vec ? LD_GEMM_VEC : LD_ANY, p, (cudaStream_t)stream);
+  const int load = vec ? LD_GEMM_VEC : LD_ANY;
+  // the overflow masks in sequential and chunk-16 order come from the packed kernel (tile override 3 keeps the
+  // scalar tracking kernel, for tests and comparisons); everything else from the scalar one
+  const bool packed = ste == LBA_STE_OF && (!chunked || chunk == BK) && g_tile_override != 3;
+  const cudaError_t e = packed ? launch_ste_packed(pl.qm == QM_FLOOR_FAST ? PQ_NONE : pl.pq, chunked ? 1 : 0, load, p, (cudaStream_t)stream)
+                               : launch_ste_mask(pl.qm, ord, ste == LBA_STE_DIFF, load, p, (cudaStream_t)stream);
   return e == cudaSuccess ? LBA_OK : cuda_fail(e);
 }
 

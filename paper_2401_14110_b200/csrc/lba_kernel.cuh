@@ -84,6 +84,7 @@ struct Problem {
   float diff_a_scale;  // product-carrier A operand -> operand whose product with B is |x w| in comparison scaling
   float diff_eps1;     // eps1 in comparison scaling
   float diff_eps2;     // eps2 (a pure ratio)
+  float ste_limit;     // packed mask variant: 0.999 * R_OF / 2^(e_max + 1) = 0.999 * (1 - 2^-(M_acc + 1))
 };
 
 // ------------------------------------------------------------------ scalar building blocks
@@ -780,11 +781,20 @@ enum PackedProd { PQ_NONE = 0, PQ_MASK = 1, PQ_MASK_SAT = 2 };
 
 // RNE: nearest-even instead of floor (then PQ_MASK means "round the product to M_prod bits").  Nearest-even
 // can raise a magnitude, so the slab-level proof that the clamp is idle is not used: it always clamps.
-template <int BM, int BN, int TM, int TN, int PQ, bool RNE, int ORD, int LD>
+//
+// STE = 1 (floor, sequential or chunk-16 order): instead of the sums the kernel writes the overflow masks of the
+// straight-through estimator STE^OF (App. D; layout as in the scalar tracking kernel).  The proof that lets a
+// slab run without the clamp is the proof that none of its steps overflows, so such a slab contributes sixteen
+// 1-bits per output without looking at them; only clamped slabs and clamped folds record bits step by step.
+// Bits that must outlive a slab wait in shared memory (per thread: 16 words for the low half of a mask1
+// word, 32 words for the mask2 word in progress), so the common path keeps the forward kernel's registers.
+template <int BM, int BN, int TM, int TN, int PQ, bool RNE, int ORD, int LD, int STE = 0>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN),
-                                  ((TM * TN == 64 && ORD != ORD_CHUNK_SLAB && !RNE) || (LD == LD_ANY && !RNE && ORD != ORD_CHUNK_SLAB))
+                                  ((TM * TN == 64 && ORD != ORD_CHUNK_SLAB && !RNE) ||
+                                   ((LD == LD_ANY || STE != 0) && !RNE && ORD != ORD_CHUNK_SLAB))
                                       ? 512 / ((BM / TM) * (BN / TN)) : 1)
     lba_contract_packed_kernel(const Problem p) {
+  static_assert(STE == 0 || (!RNE && TM == 4 && TN == 8 && (ORD == ORD_SEQ || ORD == ORD_CHUNK16)), "mask variant");
   constexpr int NT = (BM / TM) * (BN / TN);
   constexpr int TX = BN / TN;
   constexpr int ROWS = BM + BN;
@@ -812,6 +822,9 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
   // neighbours are read and filled
   unsigned (*nrm)[2] = reinterpret_cast<unsigned (*)[2]>(smem_raw + sizeof(float2) * 2 * BK * BM + sizeof(float) * 2 * BK * BN);
   unsigned* tmem_slot = reinterpret_cast<unsigned*>(nrm) + 6;  // base address written by tcgen05.alloc
+  // STE: [q][tid] words, q = i * PN + j: bits of the pair's low output in the low half, of its high output above
+  uint32_t* const stash1 = reinterpret_cast<uint32_t*>(nrm) + 8;
+  uint32_t* const stash2 = stash1 + (STE ? TM * PN * NT : 0);   // [o][tid], o = i * TN + 2 * j + half
 
   const int tid = threadIdx.x;
   const int tx = tid % TX, ty = tid / TX;
@@ -876,9 +889,17 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
   // one slab of 16 k-steps; CLAMP selects whether the magnitude clamp of Eq. 2 is applied.  The clamped
   // variant is the rare one and stays a rolled loop.  In chunk-16 order the slab starts a chunk: its first
   // step adds to zero, which is a plain (exact) scaling of the product, so the sums need no clearing.
+  uint32_t hb[STE ? TM : 1][STE ? PN : 1];  // STE: the slab's bits of a clamped slab (pair layout as stash1)
   auto slab_body = [&](int buf, auto clamp_tag) {
     constexpr bool CLAMP = decltype(clamp_tag)::value;
+    constexpr bool REC = CLAMP && STE != 0;
     constexpr int UNR = (CLAMP && !RNE) ? 1 : KUNROLL;
+    if constexpr (REC) {
+#pragma unroll
+      for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < PN; ++j) hb[i][j] = 0u;
+    }
 #pragma unroll UNR
     for (int kk = 0; kk < BK; ++kk) {
       u64 a2[TM], b2[PN];
@@ -929,6 +950,10 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
           unpack2(t, lo, hi);
           lo = and_bits(lo, mask);
           hi = and_bits(hi, mask);
+          if constexpr (REC) {  // 1 where the exact sum stayed below R_OF (its cut image decides: R_OF is on the grid)
+            if (fabsf(lo) < sat) hb[i][j] |= 1u << kk;
+            if (fabsf(hi) < sat) hb[i][j] |= 0x10000u << kk;
+          }
           if (CLAMP) {
             lo = clamp_mag(lo, sat);
             hi = clamp_mag(hi, sat);
@@ -939,9 +964,11 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
   };
 
   // second hierarchy: T <- Q_acc(C + T), C <- 0.  With CLAMP the largest |T| is returned as well.
+  uint32_t cb = 0xFFFFFFFFu;  // STE: bit o = 1 where the fold just done stayed below R_OF, o = i * TN + 2 * j + half
   auto close_chunk = [&](auto clamp_tag) -> float {
     constexpr bool CLAMP = decltype(clamp_tag)::value;
     float mx = 0.0f;
+    if constexpr (STE != 0) cb = CLAMP ? 0u : 0xFFFFFFFFu;
 #pragma unroll
     for (int i = 0; i < TM; ++i)
 #pragma unroll
@@ -955,6 +982,10 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
           unpack2(add2_rz_ftz(acc1[i][j], t2), lo, hi);
           lo = and_bits(lo, mask);
           hi = and_bits(hi, mask);
+        }
+        if constexpr (CLAMP && STE != 0) {
+          if (fabsf(lo) < sat) cb |= 1u << (i * TN + 2 * j);
+          if (fabsf(hi) < sat) cb |= 2u << (i * TN + 2 * j);
         }
         if (CLAMP) {
           lo = clamp_mag(lo, sat);
@@ -1046,6 +1077,90 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
   }
   __syncthreads();
 
+  // ---- STE bookkeeping (see the kernel's header comment)
+  bool low_fast = true;    // the even slab of the mask1 word in progress ran without the clamp
+  bool s2_active = false;  // the mask2 word in progress lives in stash2 (one of its folds was clamped)
+  const int64_t W1 = (p.K + 31) / 32;
+  const int64_t W2 = p.mask2_words;
+  // one 32-bit word for every output of the thread; word_of(i, c): micro-tile row i, column c = 2 * pair + half
+  auto emit_words = [&](uint32_t* base, int64_t words, int64_t w, auto word_of) {
+    const bool vec = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(base) & 15) == 0);
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+      const int64_t m = m0 + (i / 4) * (BM / 2) + ty * 4 + (i % 4);
+      if (m >= p.M) continue;
+#pragma unroll
+      for (int h = 0; h < TN / 4; ++h) {
+        const int64_t n = n0 + h * (BN / 2) + tx * 4;
+        uint32_t* const dst = base + (m * words + w) * p.N + n;
+        uint32_t v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) v[q] = word_of(i, h * 4 + q);
+        if (vec && n + 3 < p.N) {
+          *reinterpret_cast<uint4*>(dst) = make_uint4(v[0], v[1], v[2], v[3]);
+        } else {
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (n + q < p.N) dst[q] = v[q];
+        }
+      }
+    }
+  };
+  // after slab s: its sixteen bits per output (all ones below `keep` if it ran without the clamp, else hb)
+  // complete or start a word of mask1
+  auto ste_after_slab = [&](int s, bool cur_fast) {
+    const int64_t left = p.K - (int64_t)s * BK;
+    const uint32_t keep = left >= BK ? 0xFFFFu : ((1u << (int)left) - 1u);
+    if ((s & 1) == 0) {
+      if (s + 1 == nslab) {  // the last word has a low half only
+        if (cur_fast) emit_words(p.mask1, W1, s >> 1, [&](int, int) { return keep; });
+        else emit_words(p.mask1, W1, s >> 1, [&](int i, int c) { return (hb[i][c >> 1] >> (16 * (c & 1))) & keep; });
+      } else {
+        low_fast = cur_fast;
+        if (!cur_fast) {
+#pragma unroll
+          for (int i = 0; i < TM; ++i)
+#pragma unroll
+            for (int j = 0; j < PN; ++j) stash1[(i * PN + j) * NT + tid] = hb[i][j];
+        }
+      }
+    } else {
+      const bool lf = low_fast;
+      auto low_of = [&](int i, int c) -> uint32_t {
+        return lf ? 0xFFFFu : ((stash1[(i * PN + (c >> 1)) * NT + tid] >> (16 * (c & 1))) & 0xFFFFu);
+      };
+      if (cur_fast) emit_words(p.mask1, W1, s >> 1, [&](int i, int c) { return low_of(i, c) | (keep << 16); });
+      else emit_words(p.mask1, W1, s >> 1, [&](int i, int c) {
+        return low_of(i, c) | (((hb[i][c >> 1] >> (16 * (c & 1))) & keep) << 16);
+      });
+    }
+  };
+  // after the fold of chunk s (chunk-16 order): cb holds its bit for every output of the thread
+  auto ste_after_fold = [&](int s) {
+    const int pos = s & 31;
+    if (!s2_active && cb != 0xFFFFFFFFu) {  // first clamped fold of this word: the earlier folds all passed
+      s2_active = true;
+      const uint32_t prev = (1u << pos) - 1u;
+#pragma unroll
+      for (int o = 0; o < TM * TN; ++o) stash2[o * NT + tid] = prev;
+    }
+    if (s2_active) {
+#pragma unroll
+      for (int o = 0; o < TM * TN; ++o)
+        if ((cb >> o) & 1u) stash2[o * NT + tid] |= 1u << pos;
+    }
+    if (pos == 31 || s + 1 == nslab) {
+      const uint32_t ones = pos == 31 ? 0xFFFFFFFFu : ((2u << pos) - 1u);
+      if (s2_active) emit_words(p.mask2, W2, s >> 5, [&](int i, int c) { return stash2[(i * TN + c) * NT + tid]; });
+      else emit_words(p.mask2, W2, s >> 5, [&](int, int) { return ones; });
+      s2_active = false;
+    }
+  };
+
+  // a slab (or fold) whose sums provably stay below `lim` * 2^(e_max + 1) runs without the clamp: below 2^(e_max + 1)
+  // the mantissa mask alone respects R_OF.  The mask variant needs more, namely that no sum reaches R_OF itself
+  // (a sum in [R_OF, 2^(e_max + 1)) needs no clamp but is an overflow), so its limit is R_OF / 2^(e_max + 1)
+  const float lim = STE != 0 ? p.ste_limit : 0.999f;
   float u = 0.0f;   // upper bound of max |acc1| of this thread, as a fraction of 2^(e_max + 1)
   float u2 = 0.0f;  // chunk-16 order: the same for the second-level sums
   int slabs_in_chunk = 0;
@@ -1071,11 +1186,12 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
       }
     } else if (CH16) {
       // the chunk starts from zero, so the CTA-wide bound alone decides (same value in every thread)
-      if (grow < 0.999f) slab_body(buf, std::false_type());
+      if (grow < lim) slab_body(buf, std::false_type());
       else slab_body(buf, std::true_type());
+      if constexpr (STE != 0) ste_after_slab(s, grow < lim);
       // |T + C| <= |T| + |C| <= u2 + grow: below 1 the mask alone already respects R_OF
       const bool last = T_IN_TMEM && s + 1 == nslab;  // the final T goes to registers for the epilogue
-      if (__all_sync(0xFFFFFFFFu, u2 + grow < 0.999f)) {
+      if (__all_sync(0xFFFFFFFFu, u2 + grow < lim)) {
         if (!T_IN_TMEM) close_chunk(std::false_type());
         else if (!last) close_chunk_tmem(std::false_type(), std::false_type());
         else close_chunk_tmem(std::false_type(), std::true_type());
@@ -1087,8 +1203,9 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
         else mx = close_chunk_tmem(std::true_type(), std::true_type());
         u2 = mx * p.inv_top;
       }
+      if constexpr (STE != 0) ste_after_fold(s);
     } else {
-      bool fast = __all_sync(0xFFFFFFFFu, u + grow < 0.999f);
+      bool fast = __all_sync(0xFFFFFFFFu, u + grow < lim);
       if (!fast && u > 0.0f) {  // the carried bound may just be loose: measure |acc1|
         float mx = 0.0f;
 #pragma unroll
@@ -1100,10 +1217,11 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
             mx = fmaxf(mx, fmaxf(fabsf(lo), fabsf(hi)));
           }
         u = mx * p.inv_top;
-        fast = __all_sync(0xFFFFFFFFu, u + grow < 0.999f);
+        fast = __all_sync(0xFFFFFFFFu, u + grow < lim);
       }
       if (fast) slab_body(buf, std::false_type());
       else slab_body(buf, std::true_type());
+      if constexpr (STE != 0) ste_after_slab(s, fast);
       u = fminf(u + grow, 1.0f);
       if (CHUNKED) {
         if (++slabs_in_chunk == p.chunk_slabs) {
@@ -1125,6 +1243,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
       asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_slot), "r"(TMEM_COLS) : "memory");
     }
   }
+
+  if constexpr (STE != 0) return;  // the masks are the output
 
   // ---- epilogue: back to real values, +0 for every zero, scales and bias in binary32
   float* const outz = p.out + (int64_t)blockIdx.z * p.batch_out;
@@ -1177,6 +1297,11 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
 template <int BM, int BN>
 constexpr size_t packed_smem_bytes() {
   return sizeof(float2) * 2 * BK * BM + sizeof(float) * 2 * BK * BN + sizeof(unsigned) * 8;
+}
+// the mask variant adds its two per-thread stashes (16 + 32 words for the 4x8 micro-tile)
+template <int BM, int BN, int TM, int TN>
+constexpr size_t packed_ste_smem_bytes() {
+  return packed_smem_bytes<BM, BN>() + sizeof(uint32_t) * (BM / TM) * (BN / TN) * (TM * (TN / 2) + TM * TN);
 }
 
 // Launch entry of one (quantiser mode, order mode) family; defined once per translation unit.

@@ -342,20 +342,29 @@ def test_ste_masks_match_oracle(name, ste):
     prod, acc = FORMATS[name]
     kind, e1, e2 = (lba.STE_OF, 0.0, 0.0) if ste == "of" else (lba.STE_DIFF, 2.0 ** -20, 0.25)
     zeros = ones = zeros2 = 0
-    for (M, N, K) in ((1, 1, 1), (70, 45, 37), (66, 67, 160), (33, 129, 1000)):
+    for (M, N, K) in ((1, 1, 1), (70, 45, 37), (66, 67, 160), (33, 129, 1000), (130, 68, 1120)):
         for regime in (0, 1, 2, 3):
             A, B = _overflow_case(M, N, K, regime, 100 * regime + K + 7)
             for order, chunk in STE_ORDERS:
-                g1, g2 = lba.lba_gemm_ste_mask(A.to(DEV), B.to(DEV), prod, acc, order, chunk, kind, e1, e2)
                 w1, w2 = orc.gemm_ste_mask(A.numpy(), B.numpy(), prod.as_tuple(), acc.as_tuple(), order, chunk,
                                            orc.STE_OF if ste == "of" else orc.STE_DIFF, e1, e2)
-                what = f"{name} {ste} {M}x{N}x{K} regime {regime} order {order} chunk {chunk}"
-                bad = np.argwhere(_u32(g1) != w1)
-                assert bad.size == 0, f"{what}: mask1 differs in {len(bad)} words, first at {bad[0]}"
-                assert (g2 is None) == (w2 is None)
+                # the overflow masks in sequential and chunk-16 order come from the packed kernel by default and
+                # from the scalar tracking kernel under tile override 3: both must give the oracle's bits
+                both = ste == "of" and (order == SEQ or chunk == 16)
+                for override in ((-1, 3) if both else (-1,)):
+                    lba.set_tile_override(override)
+                    try:
+                        g1, g2 = lba.lba_gemm_ste_mask(A.to(DEV), B.to(DEV), prod, acc, order, chunk, kind, e1, e2)
+                    finally:
+                        lba.set_tile_override(-1)
+                    what = f"{name} {ste} {M}x{N}x{K} regime {regime} order {order} chunk {chunk} override {override}"
+                    bad = np.argwhere(_u32(g1) != w1)
+                    assert bad.size == 0, f"{what}: mask1 differs in {len(bad)} words, first at {bad[0]}"
+                    assert (g2 is None) == (w2 is None)
+                    if w2 is not None:
+                        bad = np.argwhere(_u32(g2) != w2)
+                        assert bad.size == 0, f"{what}: mask2 differs in {len(bad)} words, first at {bad[0]}"
                 if w2 is not None:
-                    bad = np.argwhere(_u32(g2) != w2)
-                    assert bad.size == 0, f"{what}: mask2 differs in {len(bad)} words, first at {bad[0]}"
                     zeros2 += int(w2.size * 32 - np.unpackbits(w2.view(np.uint8)).sum())
                 n1 = int(np.unpackbits(w1.view(np.uint8)).sum())
                 ones += n1
