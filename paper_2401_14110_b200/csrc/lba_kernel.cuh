@@ -1106,6 +1106,30 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
       }
     }
   };
+  // the same word for every output of the thread (the common case: nothing overflowed); a rolled loop, to keep
+  // the hot path short
+  auto emit_const = [&](uint32_t* base, int64_t words, int64_t w, uint32_t value) {
+    const bool vec = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(base) & 15) == 0);
+    const uint4 v4 = make_uint4(value, value, value, value);
+    uint32_t* row = base + ((m0 + ty * 4) * words + w) * p.N + n0 + tx * 4;
+    const int64_t pitch = words * p.N;
+#pragma unroll 1
+    for (int i = 0; i < TM; ++i, row += pitch) {
+      if (m0 + ty * 4 + i >= p.M) break;
+#pragma unroll
+      for (int h = 0; h < TN / 4; ++h) {
+        const int64_t n = n0 + h * (BN / 2) + tx * 4;
+        uint32_t* const dst = row + h * (BN / 2);
+        if (vec && n + 3 < p.N) {
+          *reinterpret_cast<uint4*>(dst) = v4;
+        } else {
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (n + q < p.N) dst[q] = value;
+        }
+      }
+    }
+  };
   // after slab s: its sixteen bits per output (all ones below `keep` if it ran without the clamp, else hb)
   // complete or start a word of mask1
   auto ste_after_slab = [&](int s, bool cur_fast) {
@@ -1113,7 +1137,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
     const uint32_t keep = left >= BK ? 0xFFFFu : ((1u << (int)left) - 1u);
     if ((s & 1) == 0) {
       if (s + 1 == nslab) {  // the last word has a low half only
-        if (cur_fast) emit_words(p.mask1, W1, s >> 1, [&](int, int) { return keep; });
+        if (cur_fast) emit_const(p.mask1, W1, s >> 1, keep);
         else emit_words(p.mask1, W1, s >> 1, [&](int i, int c) { return (hb[i][c >> 1] >> (16 * (c & 1))) & keep; });
       } else {
         low_fast = cur_fast;
@@ -1129,7 +1153,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
       auto low_of = [&](int i, int c) -> uint32_t {
         return lf ? 0xFFFFu : ((stash1[(i * PN + (c >> 1)) * NT + tid] >> (16 * (c & 1))) & 0xFFFFu);
       };
-      if (cur_fast) emit_words(p.mask1, W1, s >> 1, [&](int i, int c) { return low_of(i, c) | (keep << 16); });
+      if (cur_fast && lf) emit_const(p.mask1, W1, s >> 1, 0xFFFFu | (keep << 16));
+      else if (cur_fast) emit_words(p.mask1, W1, s >> 1, [&](int i, int c) { return low_of(i, c) | (keep << 16); });
       else emit_words(p.mask1, W1, s >> 1, [&](int i, int c) {
         return low_of(i, c) | (((hb[i][c >> 1] >> (16 * (c & 1))) & keep) << 16);
       });
@@ -1152,7 +1177,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
     if (pos == 31 || s + 1 == nslab) {
       const uint32_t ones = pos == 31 ? 0xFFFFFFFFu : ((2u << pos) - 1u);
       if (s2_active) emit_words(p.mask2, W2, s >> 5, [&](int i, int c) { return stash2[(i * TN + c) * NT + tid]; });
-      else emit_words(p.mask2, W2, s >> 5, [&](int, int) { return ones; });
+      else emit_const(p.mask2, W2, s >> 5, ones);
       s2_active = false;
     }
   };
