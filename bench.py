@@ -216,7 +216,8 @@ def describe(c):
     prod, acc = formats()
     m, n, k = c.gemm_shape
     if c.kind == "ste":
-        return "ste_mask=%s tile=64x64x16 micro=4x4 q=floor order=%s" % (STE_KIND, "chunk16" if RUN_ORDER else "seq")
+        return "ste_mask=%s tile=64x64x16 micro=%s q=floor order=%s" % (
+            STE_KIND, "4x8 packed" if STE_KIND == "of" else "4x4 scalar", "chunk16" if RUN_ORDER else "seq")
     vec = (c.x.shape[-1] % 16 == 0) if c.kind == "conv" else (k % 16 == 0)
     return lba.describe_plan(m, n, k, prod, acc, ORDER_CHUNKED, 16, is_conv=c.kind == "conv", vec_ok=vec)
 
@@ -398,12 +399,14 @@ def main():
     mhz = clocks["sm_mhz"] or max_mhz
     slots = issue_slots_per_mac(RUN_ORDER == 1, 16)
     mix = "0.5 FMUL2 + 0.5 FFMA2 + 1 LOP3, plus 2.5 per output per chunk of 16"
-    if STE_KIND is not None:
-        # scalar tracking kernel: multiply, add (toward zero), mantissa mask, compare with R_OF, clamp, bit insert;
-        # the difference estimator adds the rescaled sum, the subtraction, |x w|, + eps1, * eps2
-        slots = (6.0 if STE_KIND == "of" else 11.0) + (slots - ISSUE_SLOTS_PER_MAC_LEVEL1)
-        mix = ("FMUL + FFMA + LOP3 + FSETP + FMNMX + bit insert" if STE_KIND == "of" else
-               "FMUL + FFMA + LOP3 + FMNMX + 3 FMUL + 2 FADD + FSETP + bit insert") + ", scalar, plus the chunk folds"
+    if STE_KIND == "of":
+        # the packed kernel: slabs proved free of overflow cost what the forward pass costs, the mask words are constants
+        mix += "; the overflow mask of a slab that provably cannot overflow needs no per-step work"
+    elif STE_KIND == "diff":
+        # scalar tracking kernel: multiply, add (toward zero), mantissa mask, clamp, the rescaled sum, the subtraction,
+        # |x w|, + eps1, * eps2, compare, bit insert
+        slots = 11.0 + (slots - ISSUE_SLOTS_PER_MAC_LEVEL1)
+        mix = "FMUL + FFMA + LOP3 + FMNMX + 3 FMUL + 2 FADD + FSETP + bit insert, scalar, plus the chunk folds"
     peak = sm_count * ISSUE_LANES_PER_SM_CLK * max_mhz * 1e6 / slots / 1e9
     achieved = dom["macs"] / (dom["ms"] * 1e-3) / 1e9
     roofline = {
