@@ -102,7 +102,7 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
   const int kp = p_flush ? pf->bias - 126 : -108;  // carrier = value * 2^kp; 2^-18 * 2^-108 is still normal
   const double p_rof = r_of(pf);
   // nearest-even can carry a value in the last half step below R_OF past it, so reachability
-  // is judged with that margin; floor never increases a magnitude
+  // is assessed with that margin; floor never increases a magnitude
   const bool p_sat = p_rof <= kMaxProduct * (nearest ? 1.0 + std::ldexp(1.0, -pf->man_bits - 1) : 1.0);
   const bool p_round = pf->man_bits < 7;  // an E4M3 product has at most 8 significant bits
   const int p_emax = (1 << pf->exp_bits) - pf->bias - 1;
