@@ -49,9 +49,34 @@ def _round(v: Fraction, nearest: bool) -> int:
     return fl
 
 
+def fixed_range(B, b):
+    """(R_min, R_max) of Eq. 1."""
+    return -Fraction(2) ** (B - b - 1), Fraction(2) ** (-b) * (2 ** (B - 1) - 1)
+
+
+def quantise_fixed(fmt, x) -> Fraction:
+    """Q^FIXED_{B,b}(x), Eq. 1, cases in the printed order, Round = floor; fmt = (B, 0, b, 0, flags) and flags bit1
+    asks for two's-complement wrap-around (modulo 2^B) instead of the two saturating cases."""
+    B, E, b, rounding, flags = fmt
+    assert E == 0 and rounding == 0
+    x = Fraction(x)
+    lo, hi = fixed_range(B, b)
+    if flags & 2:
+        n = math.floor(x * Fraction(2) ** b)
+        n = (n + 2 ** (B - 1)) % 2 ** B - 2 ** (B - 1)
+        return Fraction(n) / Fraction(2) ** b
+    if x <= lo:
+        return lo
+    if x >= hi:
+        return hi
+    return Fraction(math.floor(x * Fraction(2) ** b)) / Fraction(2) ** b
+
+
 def quantise(fmt, x) -> Fraction:
-    """Q^FLOAT_{M,E,b}(x), Eq. 2, cases in the printed order; zero is +0."""
+    """Q^FLOAT_{M,E,b}(x), Eq. 2, cases in the printed order; zero is +0.  E = 0 selects Eq. 1."""
     M, E, b, rounding, flags = fmt
+    if E == 0:
+        return quantise_fixed(fmt, x)
     x = Fraction(x)
     if x == 0:
         return Fraction(0)

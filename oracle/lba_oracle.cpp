@@ -62,6 +62,10 @@ struct lbo_fmt {
   int32_t rounding;  // 0 = floor on magnitude, 1 = nearest, ties to even
   int32_t flags;     // bit0: 1 = underflow flush on (Eq. 2), 0 = "excluding underflow"
 };
+// exp_bits = 0 selects the fixed-point quantiser of Eq. 1 instead: man_bits = B (all bits, sign included),
+// bias = b, rounding 0 = floor (toward minus infinity, the plain reading of "Floor" for a two's-complement
+// number), flags bit1: 1 = wrap around modulo 2^B (the integer accumulators of the WrapNet comparison, Sec. 2.2)
+// instead of saturating at R_min / R_max.
 
 enum {
   LBO_OK = 0,
@@ -204,10 +208,27 @@ struct Fmt {
   bool nearest;    // else floor on the magnitude
   bool underflow;  // the |x| < R_UF -> 0 branch of Eq. 2 is active
   Dy r_of;         // R_OF = 2^(2^E - b - 1) * (2 - 2^-M)
+  bool fixed;      // Eq. 1 instead of Eq. 2: B = M bits in all, bias b
+  bool wrap;       // fixed point: modulo 2^B instead of saturation
 };
 
 int make_fmt(const lbo_fmt* f, Fmt* out) {
   if (!f) return LBO_ERR_ARG;
+  out->fixed = false;
+  out->wrap = false;
+  if (f->exp_bits == 0) {  // Eq. 1
+    if (f->man_bits < 2 || f->man_bits > 32 || f->rounding != 0) return LBO_ERR_FORMAT;
+    if (f->bias < -64 || f->bias > 64) return LBO_ERR_FORMAT;
+    out->fixed = true;
+    out->wrap = (f->flags & 2) != 0;
+    out->M = f->man_bits;
+    out->E = 0;
+    out->b = f->bias;
+    out->nearest = false;
+    out->underflow = false;
+    out->r_of = kZero;
+    return LBO_OK;
+  }
   if (f->man_bits < 1 || f->man_bits > 52) return LBO_ERR_FORMAT;
   if (f->exp_bits < 1 || f->exp_bits > 10) return LBO_ERR_FORMAT;
   if (f->rounding != 0 && f->rounding != 1) return LBO_ERR_FORMAT;
@@ -224,8 +245,42 @@ int make_fmt(const lbo_fmt* f, Fmt* out) {
   return LBO_OK;
 }
 
+// Q^FIXED_{B,b}(x) of Eq. 1 with Round = floor: 2^-b * floor(x * 2^b), held to [R_min, R_max] =
+// [-2^(B-1), 2^(B-1) - 1] * 2^-b by saturation (Eq. 1) or, with `wrap`, by two's-complement wrap-around.
+// |x| here is far below 2^100 (sums of bounded terms), so the integer fits the carrier.
+Dy quantise_fixed(const Fmt& f, const Dy& x) {
+  if (x.mag == 0) return kZero;
+  typedef __int128 i128;
+  const int sh = x.ex + f.b;  // x * 2^b = mag * 2^sh
+  i128 v;
+  if (sh >= 0) {
+    const int room = 120 - bit_length(x.mag);
+    u128 q = sh <= room ? (x.mag << sh) : (((u128)1) << 120);  // beyond every admitted range: saturates below
+    if (f.wrap && sh > room) q = sh >= 128 ? 0 : (x.mag << sh);  // modulo 2^B only the low bits matter (B <= 32)
+    v = x.neg ? -(i128)q : (i128)q;
+  } else {
+    const int s = -sh;
+    u128 q = s >= 128 ? 0 : (x.mag >> s);
+    const bool rem = s >= 128 ? true : ((x.mag & ((((u128)1) << s) - 1)) != 0);
+    if (x.neg && rem) q += 1;  // floor of a negative non-integer moves away from zero
+    v = x.neg ? -(i128)q : (i128)q;
+  }
+  const i128 lo = -(((i128)1) << (f.M - 1)), hi = (((i128)1) << (f.M - 1)) - 1, span = ((i128)1) << f.M;
+  if (f.wrap) {
+    i128 r = (v - lo) % span;
+    if (r < 0) r += span;
+    v = r + lo;
+  } else {
+    v = v < lo ? lo : (v > hi ? hi : v);
+  }
+  if (v == 0) return kZero;
+  Dy r = {v < 0, (u128)(v < 0 ? -v : v), -f.b};
+  return normalised(r);
+}
+
 // Q^FLOAT_{M,E,b}(x), cases in the order Eq. 2 lists them.
 Dy quantise(const Fmt& f, const Dy& x) {
+  if (f.fixed) return quantise_fixed(f, x);
   if (x.mag == 0) return kZero;
   Dy sat = f.r_of;
   sat.neg = x.neg;
@@ -567,6 +622,7 @@ int lbo_gemm_last_overflow(const uint8_t* A, const uint8_t* B, int64_t M, int64_
   const float one = 1.0f;
   int st = fill_gemm(&g, A, B, &one, 1, &one, 1, nullptr, M, N, K, pf, af, LBO_ORDER_SEQUENTIAL, 1);
   if (st != LBO_OK) return st;
+  if (g.prod.fixed || g.acc.fixed) return LBO_ERR_FORMAT;  // the estimators are defined on Eq. 2
   if (!last && M * N > 0) return LBO_ERR_ARG;
   return parallel_items(M, nthreads, [&](int64_t m) {
     for (int64_t n = 0; n < N; ++n) {
@@ -593,6 +649,7 @@ int lbo_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, 
   int st = fill_gemm(&g, A, B, &one, 1, &one, 1, nullptr, M, N, K, pf, af, order, chunk);
   if (st != LBO_OK) return st;
   if (kind != LBO_STE_OF && kind != LBO_STE_DIFF) return LBO_ERR_ARG;
+  if (g.prod.fixed || g.acc.fixed) return LBO_ERR_FORMAT;  // the estimators are defined on Eq. 2
   if (kind == LBO_STE_DIFF && !(eps1 > 0.0f && eps2 > 0.0f)) return LBO_ERR_ARG;
   const bool chunked = order == LBO_ORDER_CHUNKED;
   const int64_t W1 = (K + 31) / 32;

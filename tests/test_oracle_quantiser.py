@@ -193,4 +193,88 @@ def test_format_errors():
     with pytest.raises(orc.OracleError):
         orc.quantise((7, 4, 8, 2, 1), 1.0)
     with pytest.raises(orc.OracleError):
-        orc.quantise((7, 0, 8, 0, 1), 1.0)
+        orc.quantise((7, 11, 8, 0, 1), 1.0)          # (E = 0 is no error any more: it selects Eq. 1)
+
+
+# ---------------------------------------------------------------- Eq. 1: the fixed-point quantiser
+def test_fixed_point_hand_worked_values(golden_dir):
+    for B, b, wrap, x, want in _rows(os.path.join(golden_dir, "eq1_fixed_point.txt")):
+        fmt = (int(B), 0, int(b), 0, 2 if wrap == "1" else 0)
+        assert orc.quantise(fmt, float(x)) == float(want), (fmt, x)
+        assert ex.quantise(fmt, Fraction(x)) == Fraction(want), (fmt, x)
+
+
+def test_fixed_point_range_closed_forms_and_invariants():
+    rng = np.random.default_rng(3)
+    for B, b in ((8, 0), (12, 4), (8, 2), (6, -2), (16, 7), (24, 5)):
+        lo, hi = ex.fixed_range(B, b)
+        assert lo == -Fraction(2) ** (B - b - 1) and hi == Fraction(2 ** (B - 1) - 1, 1) / Fraction(2) ** b
+        fmt = (B, 0, b, 0, 0)
+        assert orc.quantise(fmt, 1e30) == float(hi) and orc.quantise(fmt, -1e30) == float(lo)
+        xs = np.sort(rng.uniform(float(lo) * 1.2, float(hi) * 1.2, 400))
+        ys = np.array([orc.quantise(fmt, float(x)) for x in xs])
+        assert (np.diff(ys) >= 0).all()                                   # monotone
+        assert all(orc.quantise(fmt, float(y)) == y for y in ys)          # idempotent
+        inside = (xs > float(lo)) & (xs < float(hi))
+        err = xs[inside] - ys[inside]
+        assert (err >= 0).all() and (err < 2.0 ** -b).all()               # floor: 0 <= x - Q(x) < 2^-b
+        assert all(float(ex.quantise(fmt, Fraction(float(x)))) == y for x, y in zip(xs, ys))
+        # wrap-around agrees with saturation inside the range and is periodic with period 2^(B-b)
+        wfmt = (B, 0, b, 0, 2)
+        for x in xs[inside][::20]:
+            assert orc.quantise(wfmt, float(x)) == orc.quantise(fmt, float(x))
+            assert orc.quantise(wfmt, float(x) + 2.0 ** (B - b)) == orc.quantise(fmt, float(x))
+
+
+def test_fixed_point_integer_accumulator_against_numpy_integers():
+    # b = 0: Q is integer arithmetic.  Saturation: a Python-integer loop with a clamp after every addition.
+    # Wrap-around: reduction modulo 2^B is a ring homomorphism, so the result is the exact integer dot product
+    # wrapped once, whatever the order of accumulation.
+    from paper_2401_14110_b200 import synth
+    A = synth.small_integer_codes((6, 70), 21, max_abs=15).numpy()
+    Bm = synth.small_integer_codes((5, 70), 22, max_abs=15).numpy()
+    av = synth.e4m3_decode(torch.from_numpy(A)).numpy().astype(np.int64)
+    bv = synth.e4m3_decode(torch.from_numpy(Bm)).numpy().astype(np.int64)
+    one = np.ones(1, np.float32)
+    exact = av @ bv.T
+    for Bbits in (8, 10, 12, 16):
+        lo, hi = -(1 << (Bbits - 1)), (1 << (Bbits - 1)) - 1
+        sat = (Bbits, 0, 0, 0, 0)
+        got = orc.gemm(A, Bm, one, one, None, (16, 0, 0, 0, 0), sat, 0, 1)
+        want = np.zeros_like(exact)
+        for m in range(6):
+            for n in range(5):
+                s = 0
+                for k in range(70):
+                    s = min(max(s + int(av[m, k] * bv[n, k]), lo), hi)
+                want[m, n] = s
+        assert (got == want).all()
+        wrap = (Bbits, 0, 0, 0, 2)
+        wrapped = (exact - lo) % (1 << Bbits) + lo
+        for order, chunk in ((0, 1), (1, 16), (1, 7)):
+            assert (orc.gemm(A, Bm, one, one, None, wrap, wrap, order, chunk) == wrapped).all()
+    assert (np.abs(exact) > 127).any() and (np.abs(exact) < 2047).all()
+
+
+def test_fixed_point_chain_against_exact_rationals():
+    rng = np.random.default_rng(8)
+    finite = np.array([c for c in range(256) if (c & 0x7F) != 0x7F], np.uint8)
+    one = np.ones(1, np.float32)
+    for trial in range(30):
+        K = int(rng.integers(1, 50))
+        x = finite[rng.integers(0, finite.size, K)]
+        w = finite[rng.integers(0, finite.size, K)]
+        pf = (int(rng.integers(10, 25)), 0, int(rng.integers(-2, 9)), 0, 2 * (trial % 2))
+        af = (int(rng.integers(8, 25)), 0, int(rng.integers(-4, 7)), 0, 2 * (trial % 2))
+        order, chunk = [(0, 1), (1, 16), (1, 5)][trial % 3]
+        got = orc.gemm(x[None], w[None], one, one, None, pf, af, order, chunk)[0, 0]
+        assert Fraction(float(got)) == ex.dot(pf, af, order, chunk, x, w)
+
+
+def test_fixed_point_format_errors():
+    for bad in ((1, 0, 0, 0, 0), (33, 0, 0, 0, 0), (8, 0, 0, 1, 0), (8, 0, 100, 0, 0)):
+        with pytest.raises(orc.OracleError):
+            orc.quantise(bad, 1.0)
+    x = np.full((1, 4), 0x48, np.uint8)
+    with pytest.raises(orc.OracleError):     # the estimators are defined for the floating-point accumulator
+        orc.gemm_last_overflow(x, x, (12, 0, 0, 0, 0), (12, 0, 0, 0, 0))
