@@ -55,7 +55,15 @@ typedef struct {
 } lba_fmt;
 
 enum { LBA_ROUND_FLOOR = 0, LBA_ROUND_NEAREST_EVEN = 1 };
-enum { LBA_FLAG_UNDERFLOW = 1 };
+enum { LBA_FLAG_UNDERFLOW = 1, LBA_FLAG_WRAP = 2 };
+
+/* exp_bits = 0 selects the fixed-point quantiser Q^FIXED_{B,b} of Eq. 1 (Sec. 2.1) instead, for both formats of a
+ * call or for neither (else LBA_ERR_FORMAT): man_bits = B, the number of bits including the sign, 2..24; bias = b
+ * (product format: -64..12, accumulator: -64..64); rounding must be LBA_ROUND_FLOOR, which here is floor toward
+ * minus infinity: Q(v) = 2^-b floor(v 2^b), held to [R_min, R_max] = [-2^(B-1), 2^(B-1) - 1] 2^-b by saturation as
+ * in Eq. 1 or, with flags bit1 LBA_FLAG_WRAP, by two's-complement wrap-around (the integer accumulators that
+ * Sec. 2.2 cites).  lba_gemm, lba_gemm_batched, lba_conv2d and the host-buffer variants accept such formats (an
+ * integer-only inner loop); the straight-through-estimator entry points do not. */
 enum { LBA_ORDER_SEQUENTIAL = 0, LBA_ORDER_CHUNKED = 1 };
 
 enum {

@@ -25,6 +25,7 @@ cudaError_t read_umma_error(int* code);
 cudaError_t launch_last_overflow(int qm, int load, const Problem& p, cudaStream_t stream);
 cudaError_t launch_ste_mask(int qm, int ord, int diff, int load, const Problem& p, cudaStream_t stream);
 cudaError_t launch_ste_packed(int pq, int chunk16, int load, const Problem& p, cudaStream_t stream);
+cudaError_t launch_fixed(int ord, int load, const Problem& p, cudaStream_t stream);
 
 namespace {
 
@@ -67,6 +68,10 @@ struct Plan {
   int chunk_slabs, chunk;
   int kp, ka, sx;   // product carrier = value * 2^kp, accumulator carrier = value * 2^ka, A operand = x * 2^sx
   double a_top;     // largest reachable accumulator magnitude (real domain)
+  // fixed-point accumulation (Eq. 1): the integer kernel's constants
+  bool fixed;
+  int fx_shift0, fx_lo_p, fx_hi_p, fx_sh_p, fx_wrap_p, fx_lo_a, fx_hi_a, fx_sh_a, fx_wrap_a, fx_dl, fx_dr;
+  float fx_unit;
 };
 
 bool fmt_ok(const lba_fmt* f) {
@@ -89,8 +94,48 @@ void fill_qconst(QConst* q, int M, float sat) {
 
 // Work out, on the host, how the two formats are carried in binary32 registers and which of the
 // branches of Eq. 2 can be reached at all from E4M3 inputs; refuse what cannot be carried exactly.
+// Eq. 1 formats (exp_bits = 0): man_bits = B, 2..24, so that every held integer converts to binary32 exactly;
+// floor only; biases for which no shift of the integer kernel can leave 32 bits.
+int make_fixed_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_t K, Plan* pl) {
+  for (const lba_fmt* f : {pf, af})
+    if (f->exp_bits != 0 || f->man_bits < 2 || f->man_bits > 24 || f->rounding != LBA_ROUND_FLOOR) return LBA_ERR_FORMAT;
+  if (order != LBA_ORDER_SEQUENTIAL && order != LBA_ORDER_CHUNKED) return LBA_ERR_ORDER;
+  if (order == LBA_ORDER_CHUNKED && chunk < 1) return LBA_ERR_ORDER;
+  // the product P * 2^(qx + qw), qx + qw in [-18, 10], is cut by a right shift of 22 - b_prod - qx - qw >= 0
+  if (pf->bias > 12 || pf->bias < -64 || af->bias > 64 || af->bias < -64) return LBA_ERR_FORMAT;
+  const int d = af->bias - pf->bias;  // product units -> accumulator units
+  if (d > 0 && (pf->man_bits - 1) + d > 30) return LBA_ERR_FORMAT;
+  std::memset(pl, 0, sizeof(*pl));
+  pl->fixed = true;
+  pl->qm = QM_FLOOR_FULL;
+  pl->fx_shift0 = 22 - pf->bias;
+  pl->fx_lo_p = -(1 << (pf->man_bits - 1));
+  pl->fx_hi_p = (1 << (pf->man_bits - 1)) - 1;
+  pl->fx_sh_p = 32 - pf->man_bits;
+  pl->fx_wrap_p = (pf->flags & LBA_FLAG_WRAP) ? 1 : 0;
+  pl->fx_lo_a = -(1 << (af->man_bits - 1));
+  pl->fx_hi_a = (1 << (af->man_bits - 1)) - 1;
+  pl->fx_sh_a = 32 - af->man_bits;
+  pl->fx_wrap_a = (af->flags & LBA_FLAG_WRAP) ? 1 : 0;
+  pl->fx_dl = d > 0 ? d : 0;
+  pl->fx_dr = d < 0 ? (-d > 31 ? 31 : -d) : 0;
+  pl->fx_unit = (float)std::ldexp(1.0, -af->bias);
+  pl->chunk = chunk;
+  if (order == LBA_ORDER_SEQUENTIAL || (int64_t)chunk >= K) {
+    pl->ord = ORD_SEQ;  // a single chunk: T = hold(C + 0) = C, already held
+  } else if (chunk % BK == 0) {
+    pl->ord = ORD_CHUNK_SLAB;
+    pl->chunk_slabs = chunk / BK;
+  } else {
+    pl->ord = ORD_CHUNK_ANY;
+  }
+  return LBA_OK;
+}
+
 int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_t K, Plan* pl) {
   if (!pf || !af) return LBA_ERR_NULL;
+  if (pf->exp_bits == 0 || af->exp_bits == 0) return make_fixed_plan(pf, af, order, chunk, K, pl);
+  pl->fixed = false;
   if (!fmt_ok(pf) || !fmt_ok(af)) return LBA_ERR_FORMAT;
   if (pf->rounding != af->rounding) return LBA_ERR_FORMAT;  // one rounding rule per FMAq unit
   if (order != LBA_ORDER_SEQUENTIAL && order != LBA_ORDER_CHUNKED) return LBA_ERR_ORDER;
@@ -272,6 +317,11 @@ void apply_plan(Problem* p, const Plan& pl) {
   p->rne_packed = pl.rne_packed;
   p->rne_k_acc = pl.rne_k_acc;
   p->rne_k_prod = pl.rne_k_prod;
+  p->fx_shift0 = pl.fx_shift0;
+  p->fx_lo_p = pl.fx_lo_p; p->fx_hi_p = pl.fx_hi_p; p->fx_sh_p = pl.fx_sh_p; p->fx_wrap_p = pl.fx_wrap_p;
+  p->fx_lo_a = pl.fx_lo_a; p->fx_hi_a = pl.fx_hi_a; p->fx_sh_a = pl.fx_sh_a; p->fx_wrap_a = pl.fx_wrap_a;
+  p->fx_dl = pl.fx_dl; p->fx_dr = pl.fx_dr;
+  p->fx_unit = pl.fx_unit;
 }
 
 bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0; }
@@ -279,6 +329,11 @@ bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15)
 int run(const Problem& p, const Plan& pl, int load, cudaStream_t stream) {
   if (p.M == 0 || p.N == 0 || p.batch == 0) return LBA_OK;
   if (p.batch > 65535) return LBA_ERR_SHAPE;
+  if (pl.fixed) {  // Eq. 1: the integer kernel, one tile shape
+    if ((p.N + 63) / 64 > 65535) return LBA_ERR_SHAPE;
+    const cudaError_t e = launch_fixed(pl.ord, load, p, stream);
+    return e == cudaSuccess ? LBA_OK : cuda_fail(e);
+  }
   if (g_tile_override == TILE_UMMA) {  // the tensor-core-product kernel, where it applies
     if (pl.qm == QM_FLOOR_FAST && pl.ord == ORD_CHUNK16) {
       if ((p.N + 63) / 64 > 65535) return LBA_ERR_SHAPE;
@@ -429,7 +484,7 @@ int lba_gemm_last_overflow(const uint8_t* A, const uint8_t* B, int64_t M, int64_
   Plan pl;
   const int st = make_plan(prod_fmt, acc_fmt, LBA_ORDER_SEQUENTIAL, 1, K, &pl);
   if (st != LBA_OK) return st;
-  if (pl.qm != QM_FLOOR_FAST && pl.qm != QM_FLOOR_FULL) return LBA_ERR_FORMAT;  // floor rounding only
+  if (pl.fixed || (pl.qm != QM_FLOOR_FAST && pl.qm != QM_FLOOR_FULL)) return LBA_ERR_FORMAT;  // Eq. 2, floor rounding only
   if (M == 0 || N == 0) return LBA_OK;
   if (!last || (K > 0 && (!A || !B))) return LBA_ERR_NULL;
   if ((N + 63) / 64 > 65535) return LBA_ERR_SHAPE;
@@ -456,7 +511,7 @@ int lba_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, 
   Plan pl;
   const int st = make_plan(prod_fmt, acc_fmt, order, chunk, K, &pl);
   if (st != LBA_OK) return st;
-  if (pl.qm != QM_FLOOR_FAST && pl.qm != QM_FLOOR_FULL) return LBA_ERR_FORMAT;  // floor rounding only
+  if (pl.fixed || (pl.qm != QM_FLOOR_FAST && pl.qm != QM_FLOOR_FULL)) return LBA_ERR_FORMAT;  // Eq. 2, floor rounding only
   const bool chunked = order == LBA_ORDER_CHUNKED;
   const int64_t chunks = chunked ? (K + chunk - 1) / chunk : 0;
   Problem p;
@@ -662,6 +717,12 @@ int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, 
   const int st = make_plan(prod_fmt, acc_fmt, order, chunk, K, &pl);
   if (st != LBA_OK) return st;
   const int load = vec_ok ? (is_conv ? LD_CONV_VEC : LD_GEMM_VEC) : LD_ANY;
+  if (pl.fixed) {
+    if (buf && buf_len)
+      std::snprintf(buf, buf_len, "tile=64x64x%d micro=4x4 q=fixed order=%s load=%s grid=%lldx%lld", BK, kOrdName[pl.ord],
+                    kLdName[load], (long long)((M + 63) / 64), (long long)((N + 63) / 64));
+    return LBA_OK;
+  }
   const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, 1, pl.qm, pl.ord, load);
   const TileInfo ti = tile_info(tile);
   if (buf && buf_len)

@@ -4,6 +4,7 @@ from dataclasses import dataclass
 ROUND_FLOOR = 0          # floor on the magnitude: the paper's choice (Sec. 3)
 ROUND_NEAREST_EVEN = 1   # a parameter of the benchmark's format sweep, not the paper's choice
 FLAG_UNDERFLOW = 1       # bit0 of flags: the |x| < R_UF -> 0 branch of Eq. 2 is active
+FLAG_WRAP = 2            # bit1 of flags, fixed-point formats: two's-complement wrap-around instead of saturation
 
 ORDER_SEQUENTIAL = 0     # Eq. 8-9
 ORDER_CHUNKED = 1        # two hierarchies, Sec. 3 / App. D
@@ -52,3 +53,9 @@ def code_domain_formats(man_bits: int = 7, exp_bits: int = 4, rounding: int = RO
 
 M7E4_PAPER = (LbaFormat(7, 4, 12), LbaFormat(7, 4, 10))   # real-domain biases of the ResNet runs (Sec. 3.1)
 WIDE = LbaFormat(23, 8, 127)                               # binary32-like: nothing in Eq. 2 is reachable
+
+
+def fixed_point_format(bits: int, bias: int = 0, wrap: bool = False) -> LbaFormat:
+    """Q^FIXED_{B,b} of Eq. 1 (exp_bits = 0 selects it): B bits including the sign, integer step 2^-b, floor;
+    saturation at R_min / R_max as printed, or wrap-around."""
+    return LbaFormat(bits, 0, bias, ROUND_FLOOR, FLAG_WRAP if wrap else 0)

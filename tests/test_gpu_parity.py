@@ -6,7 +6,7 @@ import torch
 from oracle import lba_oracle as orc
 from paper_2401_14110_b200 import binding as lba
 from paper_2401_14110_b200 import synth
-from paper_2401_14110_b200 import (LbaFormat, code_domain_formats, M7E4_PAPER, WIDE, ORDER_SEQUENTIAL as SEQ,
+from paper_2401_14110_b200 import (LbaFormat, fixed_point_format, code_domain_formats, M7E4_PAPER, WIDE, ORDER_SEQUENTIAL as SEQ,
                                    ORDER_CHUNKED as CHK)
 
 pytestmark = pytest.mark.gpu
@@ -405,6 +405,66 @@ def test_ste_mask_edge_cases():
         lba.lba_gemm_ste_mask(A, B, prod, acc, CHK, 16, lba.STE_DIFF, 0.0, 0.5)
     with pytest.raises(lba.LbaError):
         lba.lba_gemm_ste_mask(A, B, prod, acc, CHK, 16, lba.STE_DIFF, 1e-45, 0.5)
+
+
+FIXED = {
+    "b12_int": (fixed_point_format(16, 0), fixed_point_format(12, 0)),                # integer accumulator, saturating
+    "b12_int_wrap": (fixed_point_format(12, 0, True), fixed_point_format(12, 0, True)),
+    "finer_product": (fixed_point_format(20, 6), fixed_point_format(16, 2)),         # product re-cut on the coarser grid
+    "coarser_product": (fixed_point_format(10, -2), fixed_point_format(14, 3)),
+    "b24": (fixed_point_format(24, 5), fixed_point_format(24, 4)),
+    "b8_wrap_acc": (fixed_point_format(16, 2), fixed_point_format(8, 1, True)),
+    "tiny": (fixed_point_format(2, 0), fixed_point_format(3, -1)),
+}
+
+
+@pytest.mark.parametrize("name", list(FIXED))
+def test_fixed_point_accumulators_match_oracle(name):
+    # Eq. 1: integer inner loop on the GPU against the exact oracle, every order, ragged shapes, three data regimes
+    prod, acc = FIXED[name]
+    for (M, N, K) in ((1, 1, 1), (70, 45, 37), (66, 67, 160), (33, 129, 500)):
+        for regime in (0, 1, 2):
+            if regime == 0:
+                A, sa, B, sb = synth.gemm_case(M, N, K, config=40 + K)
+            elif regime == 1:
+                A, B = synth.random_codes((M, K), 7 + K), synth.random_codes((N, K), 8 + K)
+                sa, sb = torch.tensor([0.37]), torch.rand(N, generator=torch.Generator().manual_seed(K)) + 0.5
+            else:
+                A, B = synth.small_integer_codes((M, K), 9 + K, 15), synth.small_integer_codes((N, K), 10 + K, 15)
+                sa, sb = torch.ones(1), torch.ones(1)
+            bias = torch.randn(N, generator=torch.Generator().manual_seed(3 * K)) if regime == 1 else None
+            for order, chunk in STE_ORDERS:
+                got = gpu_gemm(A, B, sa, sb, bias, prod, acc, order, chunk)
+                want = ref_gemm(A, B, sa, sb, bias, prod, acc, order, chunk)
+                assert_bit_equal(got, want, f"{name} {M}x{N}x{K} regime {regime} order {order} chunk {chunk}")
+
+
+def test_fixed_point_conv_batched_and_errors():
+    prod, acc = FIXED["finer_product"]
+    for case in CONV_CASES[:4]:
+        b, h, w, cin, cout, kh, kw, stride, pad = case
+        x = synth.random_codes((b, h, w, cin), 31)
+        wt = synth.random_codes((cout, kh, kw, cin), 32)
+        one = torch.ones(1)
+        got = lba.lba_conv2d(x.to(DEV), wt.to(DEV), one.to(DEV), one.to(DEV), None, stride, pad, prod, acc, CHK, 16)
+        want = orc.conv2d(x.numpy(), wt.numpy(), 1.0, 1.0, None, stride, pad, prod.as_tuple(), acc.as_tuple(), CHK, 16)
+        assert_bit_equal(got, want, f"fixed-point conv {case}")
+    A = synth.random_codes((3, 20, 48), 41).to(DEV)
+    B = synth.random_codes((3, 30, 48), 42).to(DEV)
+    one = torch.ones(1, device=DEV)
+    got = lba.lba_gemm_batched(A, B, one, one, None, prod, acc, SEQ, 1)
+    for z in range(3):
+        want = orc.gemm(A[z].cpu().numpy(), B[z].cpu().numpy(), 1.0, 1.0, None, prod.as_tuple(), acc.as_tuple(), SEQ, 1)
+        assert_bit_equal(got[z], want, f"fixed-point batched problem {z}")
+    assert "q=fixed" in lba.describe_plan(64, 64, 64, prod, acc, CHK, 16)
+    a2, b2 = A[0], B[0]
+    for bad in ((prod, M7E4_PAPER[1]), (M7E4_PAPER[0], acc), (fixed_point_format(25, 0), acc),
+                (LbaFormat(12, 0, 0, 1, 0), acc), (fixed_point_format(16, 13), acc),
+                (fixed_point_format(24, 0), fixed_point_format(24, 8))):
+        with pytest.raises(lba.LbaError):
+            lba.lba_gemm(a2, b2, one, one, None, bad[0], bad[1], SEQ, 1)
+    with pytest.raises(lba.LbaError):
+        lba.lba_gemm_ste_mask(a2, b2, prod, acc, SEQ, 1, lba.STE_OF)
 
 
 def test_zero_and_empty_shapes():
