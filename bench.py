@@ -34,6 +34,7 @@ RUN_ORDER = 1        # ORDER_CHUNKED, the paper's order; a single-GEMM workload 
 GEMM_CASE = None     # (M, N, K) when --workload gemm:MxNxK[:seq|chunk] replaces the network
 STE_KIND = None      # "of" / "diff" when --workload ste:... times the mask re-computation pass
 STE_EPS = (2.0 ** -20, 0.25)
+FIXED_POINT = None   # "sat" / "wrap" when --workload fixed:... times the fixed-point accumulator (Eq. 1)
 
 # ALU roofline for sm_100.  Per SM and clock 4 schedulers issue one warp instruction each (128 lanes), the
 # FP32 pipe retires 128 lanes and the integer/logic pipe 64.  The packed floor path needs, per emulated MAC,
@@ -72,7 +73,8 @@ def parse_args():
     ap.add_argument("--workload", default="resnet18",
                     help="resnet18 (default, the benchmark), gemm:MxNxK[:seq|chunk] (one LBA GEMM on Gaussian "
                          "operands, used for kernel profiles), bgemm:ZxMxNxK[:seq|chunk] (one batched call) or "
-                         "ste:MxNxK[:of|diff][:seq|chunk] (STE mask re-computation of one GEMM)")
+                         "ste:MxNxK[:of|diff][:seq|chunk] (STE mask re-computation of one GEMM) or "
+                         "fixed:MxNxK[:seq|chunk][:wrap] (one GEMM with 12-bit fixed-point accumulation, Eq. 1)")
     ap.add_argument("--cpu-baseline-macs", type=float, default=1.5e9,
                     help="size of the oracle sample timed for cpu_baseline (emulated MACs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -149,7 +151,12 @@ class ClockSampler:
 
 
 def formats():
-    from paper_2401_14110_b200 import code_domain_formats
+    from paper_2401_14110_b200 import code_domain_formats, fixed_point_format
+    if FIXED_POINT is not None:
+        # 12-bit fixed-point formats with the ranges of the 12-bit floating ones: products up to 2^7 * 2047 >= 448^2,
+        # sums up to 2^9 * 2047 (R_OF of the M7E4 accumulator is 1044480)
+        wrap = FIXED_POINT == "wrap"
+        return fixed_point_format(12, -7, wrap), fixed_point_format(12, -9, wrap)
     return code_domain_formats(7, 4)
 
 
@@ -300,7 +307,7 @@ def reference_arm(args):
 
 
 def main():
-    global WORKLOAD, RUN_ORDER, GEMM_CASE, STE_KIND
+    global WORKLOAD, RUN_ORDER, GEMM_CASE, STE_KIND, FIXED_POINT
     args = parse_args()
     if args.workload.startswith("bgemm:"):
         parts = args.workload.split(":")
@@ -315,6 +322,14 @@ def main():
         GEMM_CASE = tuple(int(v) for v in parts[1].lower().split("x"))
         RUN_ORDER = 0 if (len(parts) > 2 and parts[2].startswith("seq")) else 1
         WORKLOAD = "single_lba_gemm_%dx%dx%d_m7e4_%s" % (GEMM_CASE + ("sequential" if RUN_ORDER == 0 else "chunk16",))
+    elif args.workload.startswith("fixed:"):
+        # fixed:MxNxK[:seq|chunk][:wrap]: one GEMM with 12-bit fixed-point product and accumulator formats
+        parts = args.workload.split(":")
+        GEMM_CASE = tuple(int(v) for v in parts[1].lower().split("x"))
+        FIXED_POINT = "wrap" if "wrap" in parts[2:] else "sat"
+        RUN_ORDER = 0 if "seq" in parts[2:] else 1
+        WORKLOAD = "fixed12_%s_gemm_%dx%dx%d_%s" % ((FIXED_POINT,) + GEMM_CASE + ("sequential" if RUN_ORDER == 0 else "chunk16",))
+        args.no_e2e = args.no_cpu_baseline = True      # kernel timing only for this workload
     elif args.workload.startswith("ste:"):
         # ste:MxNxK[:of|diff][:seq|chunk]: the mask re-computation pass of the straight-through estimators
         parts = args.workload.split(":")
@@ -402,6 +417,13 @@ def main():
     if STE_KIND == "of":
         # the packed kernel: slabs proved free of overflow cost what the forward pass costs, the mask words are constants
         mix += "; the overflow mask of a slab that provably cannot overflow needs no per-step work"
+    elif FIXED_POINT is not None:
+        # integer kernel, bound by the logic pipe (2 clocks per warp instruction): the floor (one shift), the
+        # change of grid (one shift) and the add with its hold (two add-min/max) = 4 logic-pipe instructions per
+        # step; the multiply and the shift count run beside them on the FP32/integer-multiply pipe.  These
+        # formats hold every product, so Q_prod needs no saturation.
+        slots = 8.0 + (4.0 / 16 if RUN_ORDER == 1 else 0.0)
+        mix = "2 SHF + 2 VIADDMNMX on the logic pipe at 2 clocks each; IMAD + IADD beside them; plus the chunk folds"
     elif STE_KIND == "diff":
         # scalar tracking kernel: multiply, add (toward zero), mantissa mask, clamp, the rescaled sum, the subtraction,
         # |x w|, + eps1, * eps2, compare, bit insert

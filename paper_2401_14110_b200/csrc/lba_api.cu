@@ -70,7 +70,7 @@ struct Plan {
   double a_top;     // largest reachable accumulator magnitude (real domain)
   // fixed-point accumulation (Eq. 1): the integer kernel's constants
   bool fixed;
-  int fx_shift0, fx_lo_p, fx_hi_p, fx_sh_p, fx_wrap_p, fx_lo_a, fx_hi_a, fx_sh_a, fx_wrap_a, fx_dl, fx_dr;
+  int fx_shift0, fx_lo_p, fx_hi_p, fx_sh_p, fx_hold_p, fx_lo_a, fx_hi_a, fx_sh_a, fx_wrap_a, fx_dl, fx_dr;
   float fx_unit;
 };
 
@@ -112,7 +112,9 @@ int make_fixed_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, 
   pl->fx_lo_p = -(1 << (pf->man_bits - 1));
   pl->fx_hi_p = (1 << (pf->man_bits - 1)) - 1;
   pl->fx_sh_p = 32 - pf->man_bits;
-  pl->fx_wrap_p = (pf->flags & LBA_FLAG_WRAP) ? 1 : 0;
+  // the largest product magnitude is 448^2 = 200704: if floor(448^2 * 2^b_prod) fits, Q_prod never has to hold
+  const bool p_fits = std::floor(std::ldexp(kMaxProduct, pf->bias)) <= (double)pl->fx_hi_p;
+  pl->fx_hold_p = p_fits ? 0 : ((pf->flags & LBA_FLAG_WRAP) ? 2 : 1);
   pl->fx_lo_a = -(1 << (af->man_bits - 1));
   pl->fx_hi_a = (1 << (af->man_bits - 1)) - 1;
   pl->fx_sh_a = 32 - af->man_bits;
@@ -318,7 +320,7 @@ void apply_plan(Problem* p, const Plan& pl) {
   p->rne_k_acc = pl.rne_k_acc;
   p->rne_k_prod = pl.rne_k_prod;
   p->fx_shift0 = pl.fx_shift0;
-  p->fx_lo_p = pl.fx_lo_p; p->fx_hi_p = pl.fx_hi_p; p->fx_sh_p = pl.fx_sh_p; p->fx_wrap_p = pl.fx_wrap_p;
+  p->fx_lo_p = pl.fx_lo_p; p->fx_hi_p = pl.fx_hi_p; p->fx_sh_p = pl.fx_sh_p; p->fx_hold_p = pl.fx_hold_p;
   p->fx_lo_a = pl.fx_lo_a; p->fx_hi_a = pl.fx_hi_a; p->fx_sh_a = pl.fx_sh_a; p->fx_wrap_a = pl.fx_wrap_a;
   p->fx_dl = pl.fx_dl; p->fx_dr = pl.fx_dr;
   p->fx_unit = pl.fx_unit;

@@ -4,17 +4,21 @@
 namespace lba {
 namespace {
 
-template <int ORD, int LD, bool WP, bool WA>
+template <int ORD, int LD, int HP, bool WA>
 cudaError_t launch(const Problem& p, cudaStream_t stream) {
   const dim3 grid((unsigned)((p.M + 63) / 64), (unsigned)((p.N + 63) / 64), (unsigned)p.batch);
-  lba_fixed_kernel<ORD, LD, WP, WA><<<grid, 256, 0, stream>>>(p);
+  lba_fixed_kernel<ORD, LD, HP, WA><<<grid, 256, 0, stream>>>(p);
   return cudaGetLastError();
 }
 
 template <int ORD, int LD>
 cudaError_t by_wrap(const Problem& p, cudaStream_t stream) {
-  if (p.fx_wrap_p) return p.fx_wrap_a ? launch<ORD, LD, true, true>(p, stream) : launch<ORD, LD, true, false>(p, stream);
-  return p.fx_wrap_a ? launch<ORD, LD, false, true>(p, stream) : launch<ORD, LD, false, false>(p, stream);
+  // fx_hold_p: 0 = products provably inside the product format's range, 1 = saturate, 2 = wrap around
+  switch (p.fx_hold_p) {
+    case 0: return p.fx_wrap_a ? launch<ORD, LD, 0, true>(p, stream) : launch<ORD, LD, 0, false>(p, stream);
+    case 1: return p.fx_wrap_a ? launch<ORD, LD, 1, true>(p, stream) : launch<ORD, LD, 1, false>(p, stream);
+    default: return p.fx_wrap_a ? launch<ORD, LD, 2, true>(p, stream) : launch<ORD, LD, 2, false>(p, stream);
+  }
 }
 
 template <int ORD>

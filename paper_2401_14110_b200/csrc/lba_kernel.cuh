@@ -87,7 +87,7 @@ struct Problem {
   float ste_limit;     // packed mask variant: 0.999 * R_OF / 2^(e_max + 1) = 0.999 * (1 - 2^-(M_acc + 1))
   // fixed-point accumulation (Eq. 1; the integer kernel only)
   int fx_shift0;               // 22 - b_prod
-  int fx_lo_p, fx_hi_p, fx_sh_p, fx_wrap_p;  // product: range of the integer, 32 - B, wrap-around instead of saturation
+  int fx_lo_p, fx_hi_p, fx_sh_p, fx_hold_p;  // product: range of the integer, 32 - B, 0 = never out of range / 1 = saturate / 2 = wrap
   int fx_lo_a, fx_hi_a, fx_sh_a, fx_wrap_a;  // accumulator
   int fx_dl, fx_dr;            // product units -> accumulator units: << dl then >> dr
   float fx_unit;               // 2^-b_acc

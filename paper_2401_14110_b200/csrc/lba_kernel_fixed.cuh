@@ -5,8 +5,8 @@
 // where hold() keeps the integer in [-2^(B-1), 2^(B-1) - 1] by saturation (Eq. 1) or by two's-complement
 // wrap-around (the integer accumulators of the WrapNet comparison, Sec. 2.2).  An E4M3 value is s * 2^q with an
 // integer |s| <= 15, so a product is P * 2^(qx + qw) with |P| <= 225, and floor(P * 2^t) for any integer t is one
-// arithmetic right shift of P << 22 by min(22 - t, 31) (exact: for t <= -9 the value lies in (-1, 1) and the
-// shift by 31 leaves 0 or -1).  The running sums are plain 32-bit integers in units of 2^-b_acc.
+// arithmetic right shift of P << 22 by 22 - t (exact: for t <= -9 the value lies in (-1, 1) and a shift by 31 or
+// more leaves 0 or -1).  The running sums are plain 32-bit integers in units of 2^-b_acc.
 // The host checks that none of the left shifts can leave 32 bits.
 //
 // Layout: 64 x 64 outputs per CTA, 4 x 4 per thread, 256 threads, K in slabs of 16, operands decoded once per
@@ -22,8 +22,17 @@ __device__ __forceinline__ int fx_hold(int v, int lo, int hi, int sh) {
   if (WRAP) return (v << sh) >> sh;  // sign-extend the low B bits (sh = 32 - B)
   return min(max(v, lo), hi);
 }
+// arithmetic right shift whose count may exceed 31: the PTX instruction clamps the count at 32 (all sign bits),
+// where the C++ operator would be undefined
+__device__ __forceinline__ int fx_sar(int v, int count) {
+  int d;
+  asm("shr.s32 %0, %1, %2;" : "=r"(d) : "r"(v), "r"(count));
+  return d;
+}
 
-template <int ORD, int LD, bool WRAP_P, bool WRAP_A>
+// HOLD_P: 0 = the host proved that no product leaves the product format's range (Q_prod is the floor alone),
+// 1 = saturate, 2 = wrap around.
+template <int ORD, int LD, int HOLD_P, bool WRAP_A>
 __global__ void __launch_bounds__(256) lba_fixed_kernel(const Problem p) {
   constexpr int BM = 64, BN = 64, TM = 4, TN = 4, NT = 256, TX = BN / TN;
   constexpr int ROWS = BM + BN;
@@ -93,7 +102,9 @@ __global__ void __launch_bounds__(256) lba_fixed_kernel(const Problem p) {
       }
   };
 
-  auto mac_step = [&](int buf, int kk) {
+  // UP: the accumulator's grid is finer than the product's (shift left); else equal or coarser (shift right)
+  auto mac_step = [&](int buf, int kk, auto up_tag) {
+    constexpr bool UP = decltype(up_tag)::value;
     int2 a[TM], b[TN];
     {
       const int4* src = reinterpret_cast<const int4*>(&As[buf][kk][ty * 4]);
@@ -112,9 +123,11 @@ __global__ void __launch_bounds__(256) lba_fixed_kernel(const Problem p) {
 #pragma unroll
       for (int j = 0; j < TN; ++j) {
         // Q_prod: floor(x w 2^b_prod), held to B_prod bits
-        const int np = fx_hold<WRAP_P>((a[i].x * b[j].x) >> min(a[i].y + b[j].y, 31), lo_p, hi_p, sh_p);
+        int np = fx_sar(a[i].x * b[j].x, a[i].y + b[j].y);
+        if (HOLD_P == 1) np = fx_hold<false>(np, lo_p, hi_p, sh_p);
+        if (HOLD_P == 2) np = fx_hold<true>(np, lo_p, hi_p, sh_p);
         // Q_acc: the sum on the accumulator's grid (S already lies on it, so only the product is re-cut), held
-        acc1[i][j] = fx_hold<WRAP_A>(acc1[i][j] + ((np << dl) >> dr), lo_a, hi_a, sh_a);
+        acc1[i][j] = fx_hold<WRAP_A>(acc1[i][j] + (UP ? (np << dl) : (np >> dr)), lo_a, hi_a, sh_a);
       }
   };
 
@@ -133,7 +146,8 @@ __global__ void __launch_bounds__(256) lba_fixed_kernel(const Problem p) {
       const int kmax = (int)((K - (int64_t)s * BK) < BK ? (K - (int64_t)s * BK) : BK);
 #pragma unroll 1
       for (int kk = 0; kk < kmax; ++kk) {
-        mac_step(buf, kk);
+        if (dl) mac_step(buf, kk, std::true_type());
+        else mac_step(buf, kk, std::false_type());
         if (++k_in_chunk == p.chunk) {
           close_chunk();
           k_in_chunk = 0;
@@ -141,8 +155,13 @@ __global__ void __launch_bounds__(256) lba_fixed_kernel(const Problem p) {
       }
     } else {
       // zero-padded steps past K add floor(0) = 0 to a sum that is already held: no change
+      if (dl) {
 #pragma unroll 4
-      for (int kk = 0; kk < BK; ++kk) mac_step(buf, kk);
+        for (int kk = 0; kk < BK; ++kk) mac_step(buf, kk, std::true_type());
+      } else {
+#pragma unroll 4
+        for (int kk = 0; kk < BK; ++kk) mac_step(buf, kk, std::false_type());
+      }
       if (ORD == ORD_CHUNK_SLAB) {
         if (++slabs_in_chunk == p.chunk_slabs) {
           close_chunk();
