@@ -15,6 +15,9 @@
 //     [Sec. 3, Fig. 1 (right), App. D last paragraph]
 //   * Y = X W^T with x_i = X_ki, w_i = W_li                                 [App. A]
 //   * convolution as the same dot product per output scalar                 [Eq. 3, App. A]
+//   * Q^FIXED_{B,b}: the fixed-point quantiser, floor, saturating or wrapping  [Eq. 1]
+//   * the straight-through estimators STE^OF and STE^DIFF of every FMAq step, as bit
+//     masks, and the last overflowing step of a sequential chain           [Sec. 4, App. D]
 //
 // Exactness: every intermediate value is a dyadic rational (sign, 128-bit integer
 // magnitude, power-of-two exponent).  Products and sums are formed exactly and
@@ -39,8 +42,9 @@
 //   * output scaling: out = fl32(fl32(y*sa)*sb) (+ bias), outside the FMAq unit
 //
 // Parity status: every function here is pinned by the CPU tests (closed forms of
-// Eq. 2, hand-derived chains, invariants, reduction to IEEE binary32 summation,
-// an independent exact-rational coding, brute force).  The paper's accuracy tables
+// Eq. 1 and Eq. 2, hand-derived values and chains, invariants, reduction to IEEE binary32
+// summation and to integer arithmetic, hand-worked estimator masks, an independent
+// exact-rational coding, brute force).  The paper's accuracy tables
 // need datasets and weights and are "parity unpinned".
 
 #include <cstdint>

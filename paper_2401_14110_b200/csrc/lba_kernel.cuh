@@ -327,7 +327,7 @@ struct RowLoader {
 enum { TRACK_NONE = 0, TRACK_LAST_OF = 1, TRACK_MASK_OF = 2, TRACK_MASK_DIFF = 3 };
 
 template <int BM, int BN, int TM, int TN, int QM, int ORD, int LD, int TRACK = TRACK_NONE>
-__global__ void __launch_bounds__((BM / TM) * (BN / TN)) lba_contract_kernel(const Problem p) {
+__global__ void __launch_bounds__((BM / TM) * (BN / TN), TRACK == TRACK_MASK_DIFF ? 2 : 1) lba_contract_kernel(const Problem p) {
   static_assert(TRACK == TRACK_NONE || QM == QM_FLOOR_FULL || QM == QM_FLOOR_FAST, "tracking variants use the floor quantisers");
   static_assert(TRACK != TRACK_LAST_OF || ORD == ORD_SEQ, "last-overflow index: sequential order");
   static_assert(TRACK == TRACK_NONE || ORD != ORD_CHUNK16, "tracking variants: generic orders");
