@@ -11,7 +11,7 @@ import torch
 from oracle import lba_oracle as orc
 from paper_2401_14110_b200 import binding as lba
 from paper_2401_14110_b200 import synth, workloads
-from paper_2401_14110_b200 import code_domain_formats, ORDER_SEQUENTIAL as SEQ, ORDER_CHUNKED as CHK
+from paper_2401_14110_b200 import code_domain_formats, fixed_point_format, ORDER_SEQUENTIAL as SEQ, ORDER_CHUNKED as CHK
 
 pytestmark = pytest.mark.gpu
 
@@ -137,3 +137,50 @@ def test_config5_accumulator_format_sweep_8192():
         _assert_points_equal(out, ms, ns, want, f"sweep M{m}E{e} rounding {r}")
         plans.add(lba.describe_plan(8192, 8192, 8192, prod, acc, CHK, 16).split("q=")[1].split()[0])
     assert {"floor_fast", "floor_full", "rne_full"} <= plans
+
+
+def _row_col_blocks(M, N, blocks, seed):
+    g = torch.Generator().manual_seed(seed)
+    m0 = torch.randint(0, M // 16, (blocks,), generator=g) * 16
+    n0 = torch.randint(0, N // 16, (blocks,), generator=g) * 16
+    return [(int(a), int(b)) for a, b in zip(m0, n0)]
+
+
+def test_bert_ffn_shape_ste_masks_and_fixed_point_at_full_size():
+    # the shape bench.py times for the mask re-computation and the fixed-point accumulator (BERT-base FFN-in,
+    # 4096 x 3072 x 768): seeded 16 x 16 output blocks against the oracle run on the same rows of A and B
+    M, N, K = 4096, 3072, 768
+    A, sa, B, sb = synth.gemm_case(M, N, K, config=5)
+    An, Bn = A.numpy(), B.numpy()
+    Ad, Bd, sad, sbd = A.to(DEV), B.to(DEV), sa.to(DEV), sb.to(DEV)
+    prod, acc = code_domain_formats(7, 4)
+    blocks = _row_col_blocks(M, N, 24, 99)
+    for order, chunk in ((CHK, 16), (SEQ, 1)):
+        for kind, okind, e1, e2 in ((lba.STE_OF, orc.STE_OF, 0.0, 0.0), (lba.STE_DIFF, orc.STE_DIFF, 2.0 ** -20, 0.25)):
+            g1, g2 = lba.lba_gemm_ste_mask(Ad, Bd, prod, acc, order, chunk, kind, e1, e2)
+            zeros = 0
+            for m0, n0 in blocks:
+                w1, w2 = orc.gemm_ste_mask(An[m0:m0 + 16], Bn[n0:n0 + 16], prod.as_tuple(), acc.as_tuple(), order, chunk,
+                                           okind, e1, e2)
+                got1 = g1[m0:m0 + 16, :, n0:n0 + 16].cpu().numpy().view(np.uint32)
+                assert (got1 == w1).all(), f"mask1 order {order} kind {kind} block ({m0}, {n0})"
+                if w2 is not None:
+                    got2 = g2[m0:m0 + 16, :, n0:n0 + 16].cpu().numpy().view(np.uint32)
+                    assert (got2 == w2).all(), f"mask2 order {order} kind {kind} block ({m0}, {n0})"
+                zeros += int(w1.size * 32 - np.unpackbits(w1.view(np.uint8)).sum())
+            assert kind == lba.STE_OF or zeros > 0          # swamped steps exist on Gaussian data
+            del g1, g2
+    last = lba.lba_gemm_last_overflow(Ad, Bd, prod, acc)
+    for m0, n0 in blocks:
+        want = orc.gemm_last_overflow(An[m0:m0 + 16], Bn[n0:n0 + 16], prod.as_tuple(), acc.as_tuple())
+        assert (last[m0:m0 + 16, n0:n0 + 16].cpu().numpy() == want).all()
+    # fixed-point accumulators in the formats of the benchmark's fixed-point workload
+    out = torch.empty((M, N), dtype=torch.float32, device=DEV)
+    ms, ns = synth.sample_tiles(M, N, 64, 16, 4242)
+    for wrap in (False, True):
+        pf, af = fixed_point_format(12, -7, wrap), fixed_point_format(12, -9, wrap)
+        for order in (CHK, SEQ):
+            lba.lba_gemm(Ad, Bd, sad, sbd, None, pf, af, order, 16, out=out)
+            want = orc.gemm_points(An, Bn, sa.numpy(), sb.numpy(), None, pf.as_tuple(), af.as_tuple(), order, 16, ms, ns)
+            _assert_points_equal(out, ms, ns, want, f"fixed point wrap={wrap} order {order}")
+    torch.cuda.empty_cache()
