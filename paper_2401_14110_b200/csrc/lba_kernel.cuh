@@ -920,26 +920,11 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
         const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(&Bs[buf][kk][h * (BN / 2) + tx * 4]);
         b2[h * 2 + 0] = v.x; b2[h * 2 + 1] = v.y;
       }
-#pragma unroll
-      for (int i = 0; i < TM; ++i)
-#pragma unroll
-        for (int j = 0; j < PN; ++j) {
-          u64 pr = mul2_ftz(a2[i], b2[j]);
-          if (RNE) {
-            if (PQ != PQ_NONE) {  // nearest-even on the exact product, then its saturation
-              pr = rne2_fp<false>(pr, kc_prod, neg1);
-              if (PQ == PQ_MASK_SAT) {
-                float plo, phi;
-                unpack2(pr, plo, phi);
-                pr = pack2(clamp_mag(plo, psat), clamp_mag(phi, psat));
-              }
-            }
-            const u64 ro = fma2_round_to_odd_ftz(pr, cc2, (CH16 && kk == 0) ? 0ull : acc1[i][j]);
-            float lo, hi;
-            unpack2(rne2_fp<true>(ro, kc_acc, neg1), lo, hi);
-            acc1[i][j] = pack2(clamp_mag(lo, sat), clamp_mag(hi, sat));
-            continue;
-          }
+      if constexpr (!RNE) {
+        // floor: the products of micro-tile row i + 1 are formed while row i is added and masked, so that
+        // multiplies (FP32 pipe) and masks (logic pipe) of independent outputs sit side by side in the stream
+        auto product = [&](u64 av, u64 bv) -> u64 {
+          u64 pr = mul2_ftz(av, bv);
           if (PQ != PQ_NONE) {  // floor of Eq. 2 on the exact product, then its saturation
             float plo, phi;
             unpack2(pr, plo, phi);
@@ -951,20 +936,59 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
             }
             pr = pack2(plo, phi);
           }
-          const u64 t = (CH16 && kk == 0) ? mul2_rz_ftz(pr, cc2) : fma2_rz_ftz(pr, cc2, acc1[i][j]);
+          return pr;
+        };
+        u64 pr[PN], nx[PN];
+#pragma unroll
+        for (int j = 0; j < PN; ++j) pr[j] = product(a2[0], b2[j]);
+#pragma unroll
+        for (int i = 0; i < TM; ++i) {
+          if (i + 1 < TM) {
+#pragma unroll
+            for (int j = 0; j < PN; ++j) nx[j] = product(a2[i + 1], b2[j]);
+          }
+#pragma unroll
+          for (int j = 0; j < PN; ++j) {
+            const u64 t = (CH16 && kk == 0) ? mul2_rz_ftz(pr[j], cc2) : fma2_rz_ftz(pr[j], cc2, acc1[i][j]);
+            float lo, hi;
+            unpack2(t, lo, hi);
+            lo = and_bits(lo, mask);
+            hi = and_bits(hi, mask);
+            if constexpr (REC) {  // 1 where the exact sum stayed below R_OF (its cut image decides: R_OF is on the grid)
+              if (fabsf(lo) < sat) hb[i][j] |= 1u << kk;
+              if (fabsf(hi) < sat) hb[i][j] |= 0x10000u << kk;
+            }
+            if (CLAMP) {
+              lo = clamp_mag(lo, sat);
+              hi = clamp_mag(hi, sat);
+            }
+            acc1[i][j] = pack2(lo, hi);
+          }
+          if (i + 1 < TM) {
+#pragma unroll
+            for (int j = 0; j < PN; ++j) pr[j] = nx[j];
+          }
+        }
+        continue;
+      }
+#pragma unroll
+      for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < PN; ++j) {
+          // nearest-even (the floor path has left the loop body above)
+          u64 pr = mul2_ftz(a2[i], b2[j]);
+          if (PQ != PQ_NONE) {  // nearest-even on the exact product, then its saturation
+            pr = rne2_fp<false>(pr, kc_prod, neg1);
+            if (PQ == PQ_MASK_SAT) {
+              float plo, phi;
+              unpack2(pr, plo, phi);
+              pr = pack2(clamp_mag(plo, psat), clamp_mag(phi, psat));
+            }
+          }
+          const u64 ro = fma2_round_to_odd_ftz(pr, cc2, (CH16 && kk == 0) ? 0ull : acc1[i][j]);
           float lo, hi;
-          unpack2(t, lo, hi);
-          lo = and_bits(lo, mask);
-          hi = and_bits(hi, mask);
-          if constexpr (REC) {  // 1 where the exact sum stayed below R_OF (its cut image decides: R_OF is on the grid)
-            if (fabsf(lo) < sat) hb[i][j] |= 1u << kk;
-            if (fabsf(hi) < sat) hb[i][j] |= 0x10000u << kk;
-          }
-          if (CLAMP) {
-            lo = clamp_mag(lo, sat);
-            hi = clamp_mag(hi, sat);
-          }
-          acc1[i][j] = pack2(lo, hi);
+          unpack2(rne2_fp<true>(ro, kc_acc, neg1), lo, hi);
+          acc1[i][j] = pack2(clamp_mag(lo, sat), clamp_mag(hi, sat));
         }
     }
   };
