@@ -26,6 +26,7 @@ cudaError_t launch_last_overflow(int qm, int load, const Problem& p, cudaStream_
 cudaError_t launch_ste_mask(int qm, int ord, int diff, int load, const Problem& p, cudaStream_t stream);
 cudaError_t launch_ste_packed(int pq, int chunk16, int load, const Problem& p, cudaStream_t stream);
 cudaError_t launch_fixed(int ord, int load, const Problem& p, cudaStream_t stream);
+cudaError_t launch_cluster_pair(int pq, int load, const Problem& p, cudaStream_t stream);
 
 namespace {
 
@@ -56,6 +57,7 @@ const char* const kLdName[LD_COUNT] = {"gemm_vec", "conv_vec", "any"};
 
 // Largest |x*w| of two E4M3 values and the grid every product lies on.
 constexpr double kMaxProduct = 448.0 * 448.0;  // 200704
+constexpr double kPairEff = 0.95;              // MAC rate of the cluster-pair tile relative to the plain 64x64 tile
 constexpr int kMinProductExp = -18;            // every product, hence every sum, is a multiple of 2^-18
 
 struct Plan {
@@ -258,9 +260,11 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
 // Tile choice.  All CTAs of a launch have the same work and K is never split, so the launch ends when the
 // busiest SM has run its ceil(CTAs / SMs) tiles; larger tiles spend fewer instructions per MAC (eff, measured
 // on B200 with every SM loaded), smaller ones fill the SMs more evenly.  Pick the cheapest by that model.
-int choose_tile(int64_t M, int64_t N, int64_t batch, int qm, int ord, int load) {
+// pair_ok: the call qualifies for the 64x64 tile shared by a cluster of two CTAs (TILE_PAIR)
+int choose_tile(int64_t M, int64_t N, int64_t batch, int qm, int ord, int load, bool pair_ok = false) {
   (void)qm;
   if (g_tile_override >= 0 && g_tile_override < TILE_COUNT) return g_tile_override;
+  if (g_tile_override == TILE_PAIR && pair_ok) return TILE_PAIR;
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) {
     int v = 0;
@@ -285,6 +289,13 @@ int choose_tile(int64_t M, int64_t N, int64_t batch, int qm, int ord, int load) 
       best_cost = cost;
       best = t;
     }
+  }
+  if (pair_ok) {
+    // two CTAs per 64x64 tile, each with half the chunks: twice the CTAs at half the work, a few per cent for the
+    // hand-over of the chunk sums and the cluster barrier
+    const double ctas = 2.0 * (double)((M + 63) / 64) * (double)((N + 63) / 64) * (double)batch;
+    const double cost = std::ceil(ctas / sms) * (64.0 * 64.0 / 2.0) / (eff[2] * kPairEff);
+    if (cost < best_cost) best = TILE_PAIR;
   }
   return best;
 }
@@ -343,7 +354,15 @@ int run(const Problem& p, const Plan& pl, int load, cudaStream_t stream) {
       return e == cudaSuccess ? LBA_OK : cuda_fail(e);
     }
   }
-  const int tile = choose_tile(p.M, p.N, p.batch, pl.qm, pl.ord, load);
+  const bool pair_ok = pl.ord == ORD_CHUNK16 && (pl.qm == QM_FLOOR_FAST || pl.qm == QM_FLOOR_FULL) && load != LD_ANY &&
+                       (p.qa.mask & 0xFFFFu) == 0u &&                      // at most 7 mantissa bits: bfloat16 hand-over
+                       2 * ((p.M + 63) / 64) <= 2147483647LL;
+  const int tile = choose_tile(p.M, p.N, p.batch, pl.qm, pl.ord, load, pair_ok);
+  if (tile == TILE_PAIR) {
+    if ((p.N + 63) / 64 > 65535) return LBA_ERR_SHAPE;
+    const cudaError_t e = launch_cluster_pair(pl.qm == QM_FLOOR_FAST ? PQ_NONE : pl.pq, load, p, stream);
+    return e == cudaSuccess ? LBA_OK : cuda_fail(e);
+  }
   const TileInfo ti = tile_info(tile);
   if ((p.N + ti.bn - 1) / ti.bn > 65535 || (p.M + ti.bm - 1) / ti.bm > 2147483647LL) return LBA_ERR_SHAPE;
   const cudaError_t e = kLaunch[pl.qm][pl.ord](tile, load, p, stream);
@@ -396,7 +415,7 @@ int lba_device_error(int* code) {
 int lba_last_cuda_error(void) { return g_last_cuda_error; }
 
 int lba_set_tile_override(int tile) {
-  if (tile < -1 || tile > TILE_UMMA) return LBA_ERR_SHAPE;
+  if (tile < -1 || tile > TILE_PAIR) return LBA_ERR_SHAPE;
   g_tile_override = tile;
   return LBA_OK;
 }
@@ -725,7 +744,15 @@ int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, 
                     kLdName[load], (long long)((M + 63) / 64), (long long)((N + 63) / 64));
     return LBA_OK;
   }
-  const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, 1, pl.qm, pl.ord, load);
+  const bool pair_ok = pl.ord == ORD_CHUNK16 && (pl.qm == QM_FLOOR_FAST || pl.qm == QM_FLOOR_FULL) && load != LD_ANY &&
+                       (pl.qa.mask & 0xFFFFu) == 0u;
+  const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, 1, pl.qm, pl.ord, load, pair_ok);
+  if (tile == TILE_PAIR) {
+    if (buf && buf_len)
+      std::snprintf(buf, buf_len, "tile=64x64x%d pair micro=4x8 q=%s order=%s load=%s grid=%lldx%lld", BK, kQmName[pl.qm],
+                    kOrdName[pl.ord], kLdName[load], (long long)(2 * ((M + 63) / 64)), (long long)((N + 63) / 64));
+    return LBA_OK;
+  }
   const TileInfo ti = tile_info(tile);
   if (buf && buf_len)
     std::snprintf(buf, buf_len, "tile=%dx%dx%d micro=%dx%d q=%s order=%s load=%s grid=%lldx%lld", ti.bm, ti.bn, BK,

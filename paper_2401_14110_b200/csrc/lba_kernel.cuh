@@ -293,6 +293,12 @@ struct RowLoader {
       }
       raw[l] = v;
     }
+    skip_slab(p);
+  }
+
+  // move the convolution cursors past one slab without fetching it (fetch does this itself; a CTA that
+  // handles every second slab calls it once more)
+  __device__ __forceinline__ void skip_slab(const Problem& p) {
     if (LD == LD_ANY && p.is_conv) {  // advance the run cursor by one slab
       const int run = p.KW * p.Cin;
       any_off += BK;
@@ -794,13 +800,22 @@ enum PackedProd { PQ_NONE = 0, PQ_MASK = 1, PQ_MASK_SAT = 2 };
 // 1-bits per output without looking at them; only clamped slabs and clamped folds record bits step by step.
 // Bits that must outlive a slab wait in shared memory (per thread: 16 words for the low half of a mask1
 // word, 32 words for the mask2 word in progress), so the common path keeps the forward kernel's registers.
-template <int BM, int BN, int TM, int TN, int PQ, bool RNE, int ORD, int LD, int STE = 0>
+//
+// CL = 2 (floor, chunk-16 order, accumulator mantissa of at most 7 bits): two CTAs of a thread-block cluster share
+// one output tile.  The chunk sums C_j of the first hierarchy do not depend on each other; only the folds
+// T <- Q_acc(C_j + T), one addition in sixteen, are sequential.  CTA r forms the chunk sums of the chunks j = r, r + 2,
+// ... for the whole tile and folds, in chunk order, all chunks for the column half r of every thread's micro-tile;
+// the chunk sums of the other half cross to the other CTA through distributed shared memory (as bfloat16 pairs: a
+// value with M <= 7 mantissa bits is one exactly), double buffered, with one cluster barrier per pair of chunks.
+// This doubles the CTAs of a small problem without splitting any sequential chain, and both CTAs do the same work.
+template <int BM, int BN, int TM, int TN, int PQ, bool RNE, int ORD, int LD, int STE = 0, int CL = 1>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN),
                                   ((TM * TN == 64 && ORD != ORD_CHUNK_SLAB && !RNE) ||
                                    ((LD == LD_ANY || STE != 0) && !RNE && ORD != ORD_CHUNK_SLAB))
                                       ? 512 / ((BM / TM) * (BN / TN)) : 1)
     lba_contract_packed_kernel(const Problem p) {
   static_assert(STE == 0 || (!RNE && TM == 4 && TN == 8 && (ORD == ORD_SEQ || ORD == ORD_CHUNK16)), "mask variant");
+  static_assert(CL == 1 || (CL == 2 && !RNE && STE == 0 && ORD == ORD_CHUNK16 && TM == 4), "cluster variant");
   constexpr int NT = (BM / TM) * (BN / TN);
   constexpr int TX = BN / TN;
   constexpr int ROWS = BM + BN;
@@ -834,9 +849,13 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
 
   const int tid = threadIdx.x;
   const int tx = tid % TX, ty = tid / TX;
-  const int64_t m0 = (int64_t)blockIdx.x * BM;
+  unsigned crank = 0;  // rank of this CTA in its cluster (CL = 2: 0 folds, 1 hands its chunk sums over)
+  if (CL > 1) asm("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
+  const int64_t m0 = (int64_t)(blockIdx.x / CL) * BM;
   const int64_t n0 = (int64_t)blockIdx.y * BN;
   const int nslab = (int)((p.K + BK - 1) / BK);
+  // CL = 2: chunk sums in flight from CTA 1 to CTA 0, [buffer][group of 4 pairs][thread] as uint4 of bfloat16 pairs
+  uint4* const hand = reinterpret_cast<uint4*>(reinterpret_cast<uint32_t*>(nrm) + 8);
 
   RowLoader<BM, BN, NT, LD> loader;
   loader.init(p, tid, m0, n0);
@@ -971,6 +990,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
         }
         continue;
       }
+      if constexpr (RNE) {
 #pragma unroll
       for (int i = 0; i < TM; ++i)
 #pragma unroll
@@ -990,6 +1010,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
           unpack2(rne2_fp<true>(ro, kc_acc, neg1), lo, hi);
           acc1[i][j] = pack2(clamp_mag(lo, sat), clamp_mag(hi, sat));
         }
+      }
     }
   };
 
@@ -1101,8 +1122,10 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
     tmem_wait_st();
   }
   uint4 raw[LPT];
-  if (nslab > 0) {
-    loader.fetch(p, tid, 0, raw);
+  const int s_first = CL > 1 ? (int)crank : 0;  // first slab of this CTA
+  if (CL > 1 && crank != 0) loader.skip_slab(p);
+  if (s_first < nslab) {
+    loader.fetch(p, tid, s_first, raw);
     decode_store(raw, 0, 0);
   }
   __syncthreads();
@@ -1220,6 +1243,153 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
   float u2 = 0.0f;  // chunk-16 order: the same for the second-level sums
   int slabs_in_chunk = 0;
   int cell = 0;     // s % 3
+  if constexpr (CL > 1) {
+    // ---- two CTAs per output tile (see the kernel's header comment).  Both run the same number of rounds and
+    // meet at one cluster barrier per round; nothing leaves the loop early.  CTA r forms the chunk sums of the
+    // chunks 2q + r for the whole tile, but keeps and folds the second-level sums T only for the column half r of
+    // every thread's micro-tile; the chunk sums of the other half go to the other CTA.  The work is the same on
+    // both sides: one slab and two folds of half a micro-tile per round.
+    static_assert(PN == 4, "column halves of the 4x8 micro-tile");
+    constexpr int HP = PN / 2;  // pairs per row in a column half
+    const int rounds = (nslab + CL - 1) / CL;
+    uint32_t hand_remote;  // the other CTA's hand buffer as seen from this CTA
+    asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(hand_remote) : "r"((uint32_t)__cvta_generic_to_shared(hand)), "r"(crank ^ 1u));
+    u64 T[TM][HP];
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+      for (int j = 0; j < HP; ++j) T[i][j] = 0ull;
+
+    // T <- Q_acc(C + T) for this CTA's column half H; C from the own chunk sums (acc1) or from the words received
+    auto fold = [&](auto half_tag, auto clamp_tag, const uint32_t* recv) -> float {
+      constexpr int H = decltype(half_tag)::value;
+      constexpr bool CLAMP = decltype(clamp_tag)::value;
+      float mx = 0.0f;
+#pragma unroll
+      for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < HP; ++j) {
+          const u64 c = recv ? pack2u(recv[i * HP + j] << 16, recv[i * HP + j] & 0xFFFF0000u) : acc1[i][H * HP + j];
+          float lo, hi;
+          unpack2(add2_rz_ftz(c, T[i][j]), lo, hi);
+          lo = and_bits(lo, mask);
+          hi = and_bits(hi, mask);
+          if (CLAMP) {
+            lo = clamp_mag(lo, sat);
+            hi = clamp_mag(hi, sat);
+            mx = fmaxf(mx, fmaxf(fabsf(lo), fabsf(hi)));
+          }
+          T[i][j] = pack2(lo, hi);
+        }
+      return mx;
+    };
+    // the own chunk may skip the clamp under the running bound; a received chunk is always clamped and
+    // refreshes the bound
+    auto fold_own = [&](auto half_tag, float grow) {
+      if (__all_sync(0xFFFFFFFFu, u2 + grow < lim)) {
+        fold(half_tag, std::false_type(), nullptr);
+        u2 += grow;
+      } else {
+        u2 = fold(half_tag, std::true_type(), nullptr) * p.inv_top;
+      }
+    };
+    auto fold_received = [&](auto half_tag, int q) {
+      uint32_t w[TM * HP];
+#pragma unroll
+      for (int g = 0; g < TM * HP / 4; ++g) {
+        const uint4 v = hand[((q & 1) * (TM * HP / 4) + g) * NT + tid];
+        w[g * 4 + 0] = v.x; w[g * 4 + 1] = v.y; w[g * 4 + 2] = v.z; w[g * 4 + 3] = v.w;
+      }
+      u2 = fold(half_tag, std::true_type(), w) * p.inv_top;
+    };
+    // chunk sums of the column half `other` as bfloat16 pairs (exact for M <= 7) into the other CTA's buffer
+    auto send = [&](auto other_tag, int q) {
+      constexpr int O = decltype(other_tag)::value;
+#pragma unroll
+      for (int g = 0; g < TM * HP / 4; ++g) {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int idx = g * 4 + e;
+          float lo, hi;
+          unpack2(acc1[idx / HP][O * HP + idx % HP], lo, hi);
+          w[e] = (__float_as_uint(lo) >> 16) | (__float_as_uint(hi) & 0xFFFF0000u);
+        }
+        const uint32_t dst = hand_remote + (uint32_t)(((q & 1) * (TM * HP / 4) + g) * NT + tid) * 16u;
+        asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                     "r"(w[3]) : "memory");
+      }
+    };
+
+    for (int q = 0; q < rounds; ++q) {
+      const int s = q * CL + (int)crank;
+      const bool have = s < nslab;          // only CTA 1 can run out, in the last round of an odd slab count
+      const bool more = s + CL < nslab;
+      const int buf = q & 1;
+      const int cell_next = cell == 2 ? 0 : cell + 1;
+      const int cell_clear = cell_next == 2 ? 0 : cell_next + 1;
+      if (more) {
+        loader.skip_slab(p);
+        loader.fetch(p, tid, s + CL, raw);
+      }
+      float grow = 0.0f;
+      if (have) {
+        const float na = __uint_as_float(nrm[cell][0]), nb = __uint_as_float(nrm[cell][1]);
+        if (tid < 2) nrm[cell_clear][tid] = 0u;
+        grow = sqrtf(na * nb) * 1.01f;
+        if (grow < lim) slab_body(buf, std::false_type());
+        else slab_body(buf, std::true_type());
+        if (crank == 0) send(std::integral_constant<int, 1>(), q);
+        else send(std::integral_constant<int, 0>(), q);
+      }
+      asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+      asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+      // chunk 2q (formed by CTA 0) is folded before chunk 2q + 1 (formed by CTA 1), on both sides
+      if (crank == 0) {
+        fold_own(std::integral_constant<int, 0>(), grow);
+        if (s + 1 < nslab) fold_received(std::integral_constant<int, 0>(), q);
+      } else {
+        fold_received(std::integral_constant<int, 1>(), q);
+        if (have) fold_own(std::integral_constant<int, 1>(), grow);
+      }
+      if (more) decode_store(raw, buf ^ 1, cell_next);
+      __syncthreads();
+      cell = cell_next;
+    }
+
+    // ---- epilogue of the pair: this CTA's column half
+    float* const outz = p.out + (int64_t)blockIdx.z * p.batch_out;
+    const bool vec_store = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(outz) & 15) == 0);
+    const int64_t n = n0 + (int64_t)crank * (BN / 2) + tx * 4;
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+      const int64_t m = m0 + ty * 4 + i;
+      if (m >= p.M) continue;
+      const float sa = p.sa[p.sa_per_row ? m : 0];
+      float o[4];
+#pragma unroll
+      for (int jp = 0; jp < HP; ++jp) unpack2(T[i][jp], o[jp * 2], o[jp * 2 + 1]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float y = __fmul_rn(__fmul_rn(o[j], p.un1), p.un2);
+        o[j] = (y == 0.0f) ? 0.0f : y;
+        if (n + j < p.N) {
+          const float sb = p.sb[p.sb_per_col ? n + j : 0];
+          float r = __fmul_rn(__fmul_rn(o[j], sa), sb);
+          if (p.bias) r = __fadd_rn(r, p.bias[n + j]);
+          o[j] = r;
+        }
+      }
+      if (n + 3 < p.N && vec_store) {
+        *reinterpret_cast<float4*>(outz + m * p.N + n) = make_float4(o[0], o[1], o[2], o[3]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (n + j < p.N) outz[m * p.N + n + j] = o[j];
+      }
+    }
+    return;
+  } else
   for (int s = 0; s < nslab; ++s) {
     const int buf = s & 1;
     const int cell_next = cell == 2 ? 0 : cell + 1;
@@ -1353,6 +1523,11 @@ template <int BM, int BN>
 constexpr size_t packed_smem_bytes() {
   return sizeof(float2) * 2 * BK * BM + sizeof(float) * 2 * BK * BN + sizeof(unsigned) * 8;
 }
+// the cluster variant adds the double-buffered hand-over of chunk sums (one bfloat16 per output of a column half and buffer)
+template <int BM, int BN, int TM, int TN>
+constexpr size_t packed_cluster_smem_bytes() {
+  return packed_smem_bytes<BM, BN>() + sizeof(uint32_t) * 2 * (BM / TM) * (BN / TN) * (TM * (TN / 4));
+}
 // the mask variant adds its two per-thread stashes (16 + 32 words for the 4x8 micro-tile)
 template <int BM, int BN, int TM, int TN>
 constexpr size_t packed_ste_smem_bytes() {
@@ -1367,6 +1542,7 @@ constexpr size_t packed_ste_smem_bytes() {
 struct TileInfo { int bm, bn, tm, tn; };
 constexpr int TILE_COUNT = 4;
 constexpr int TILE_UMMA = 4;  // override value that selects the tensor-core-product kernel (128 x 64 tile)
+constexpr int TILE_PAIR = 5;  // 64x64 tile shared by a cluster of two CTAs (chunk-16 order, floor, M_acc <= 7)
 __host__ inline TileInfo tile_info(int t) {
   const TileInfo tab[TILE_COUNT] = {{128, 128, 8, 8}, {128, 64, 4, 8}, {64, 64, 4, 8}, {32, 32, 4, 4}};
   return tab[t];

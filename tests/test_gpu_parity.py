@@ -467,6 +467,41 @@ def test_fixed_point_conv_batched_and_errors():
         lba.lba_gemm_ste_mask(a2, b2, prod, acc, SEQ, 1, lba.STE_OF)
 
 
+@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_paper", "m4e4", "m4e3_mnist", "m7e4_no_uf"])
+def test_cluster_pair_tile_is_exact(name):
+    # two CTAs per output tile, each taking every second chunk of 16 (tile override 5): same bits as the oracle
+    prod, acc = FORMATS[name]
+    lba.set_tile_override(5)
+    try:
+        assert "pair" in lba.describe_plan(256, 256, 256, prod, acc, CHK, 16)
+        for (M, N, K) in ((1, 1, 16), (70, 45, 32), (66, 67, 160), (33, 129, 1008), (130, 68, 1120), (64, 64, 48)):
+            for regime in (0, 1, 2, 3):
+                A, B = _overflow_case(M, N, K, regime, 50 * regime + K + 3)
+                sa = torch.tensor([0.5])
+                sb = torch.rand(N, generator=torch.Generator().manual_seed(K)) + 0.5
+                got = gpu_gemm(A, B, sa, sb, None, prod, acc, CHK, 16)
+                want = ref_gemm(A, B, sa, sb, None, prod, acc, CHK, 16)
+                assert_bit_equal(got, want, f"pair tile {name} {M}x{N}x{K} regime {regime}")
+        # convolutions with 16-byte taps
+        for case in [c for c in CONV_CASES if c[3] % 16 == 0]:
+            b, h, w, cin, cout, kh, kw, stride, pad = case
+            x = synth.random_codes((b, h, w, cin), 61) & 0x7F
+            wt = synth.random_codes((cout, kh, kw, cin), 62)
+            one = torch.ones(1)
+            got = lba.lba_conv2d(x.to(DEV), wt.to(DEV), one.to(DEV), one.to(DEV), None, stride, pad, prod, acc, CHK, 16)
+            want = orc.conv2d(x.numpy(), wt.numpy(), 1.0, 1.0, None, stride, pad, prod.as_tuple(), acc.as_tuple(), CHK, 16)
+            assert_bit_equal(got, want, f"pair tile {name} conv {case}")
+        # not eligible: falls back to the automatic choice, still exact
+        p10, a10 = FORMATS["m10e5"]
+        A, B = _overflow_case(40, 40, 64, 3, 5)
+        one = torch.ones(1)
+        assert "pair" not in lba.describe_plan(40, 40, 64, p10, a10, CHK, 16)
+        assert_bit_equal(gpu_gemm(A, B, one, one, None, p10, a10, CHK, 16), ref_gemm(A, B, one, one, None, p10, a10, CHK, 16))
+    finally:
+        lba.set_tile_override(-1)
+    assert lba.device_error() == 0
+
+
 def test_zero_and_empty_shapes():
     prod, acc = code_domain_formats(7, 4)
     one = torch.ones(1)
