@@ -223,8 +223,8 @@ int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, 
 /* Testing and tuning hook: force the CTA tile (0 = 128x128, 1 = 128x64, 2 = 64x64, 3 = 32x32
  * outputs; 4 = the experimental kernel whose products come from the tensor cores, 128x64 outputs, used only
  * for the fast floor quantiser in chunk-16 order and ignored otherwise; 5 = the 64x64 tile shared by a cluster of two
- * CTAs, each taking every second chunk, used only in chunk-16 order with floor rounding, an accumulator mantissa of at
- * most 7 bits and 16-byte loads, ignored otherwise; -1 = automatic choice, the default).  For
+ * CTAs, each taking every second chunk, used only in chunk-16 order with floor rounding and 16-byte loads, ignored
+ * otherwise; -1 = automatic choice, the default).  For
  * lba_gemm_ste_mask, 3 selects the scalar tracking kernel where the packed one would run.  Process-wide; results never
  * depend on the tile, only speed does.  Returns LBA_OK, or LBA_ERR_SHAPE for an unknown tile. */
 int lba_set_tile_override(int tile);

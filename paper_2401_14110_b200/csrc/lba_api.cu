@@ -355,7 +355,6 @@ int run(const Problem& p, const Plan& pl, int load, cudaStream_t stream) {
     }
   }
   const bool pair_ok = pl.ord == ORD_CHUNK16 && (pl.qm == QM_FLOOR_FAST || pl.qm == QM_FLOOR_FULL) && load != LD_ANY &&
-                       (p.qa.mask & 0xFFFFu) == 0u &&                      // at most 7 mantissa bits: bfloat16 hand-over
                        2 * ((p.M + 63) / 64) <= 2147483647LL;
   const int tile = choose_tile(p.M, p.N, p.batch, pl.qm, pl.ord, load, pair_ok);
   if (tile == TILE_PAIR) {
@@ -744,8 +743,7 @@ int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, 
                     kLdName[load], (long long)((M + 63) / 64), (long long)((N + 63) / 64));
     return LBA_OK;
   }
-  const bool pair_ok = pl.ord == ORD_CHUNK16 && (pl.qm == QM_FLOOR_FAST || pl.qm == QM_FLOOR_FULL) && load != LD_ANY &&
-                       (pl.qa.mask & 0xFFFFu) == 0u;
+  const bool pair_ok = pl.ord == ORD_CHUNK16 && (pl.qm == QM_FLOOR_FAST || pl.qm == QM_FLOOR_FULL) && load != LD_ANY;
   const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, 1, pl.qm, pl.ord, load, pair_ok);
   if (tile == TILE_PAIR) {
     if (buf && buf_len)

@@ -1,5 +1,5 @@
 // Chunk-16 order with two CTAs of a thread-block cluster per output tile (see lba_contract_packed_kernel, CL = 2):
-// 64x64 tile, 4x8 outputs per thread, floor quantisers, accumulator mantissa of at most 7 bits.
+// 64x64 tile, 4x8 outputs per thread, floor quantisers.
 #include "lba_kernel.cuh"
 
 namespace lba {
@@ -7,9 +7,9 @@ namespace {
 
 constexpr int BM = 64, BN = 64, TM = 4, TN = 8, CL = 2;
 
-template <int PQ, int LD>
+template <int PQ, int LD, bool H16>
 cudaError_t launch(const Problem& p, cudaStream_t stream) {
-  auto kernel = lba_contract_packed_kernel<BM, BN, TM, TN, PQ, false, ORD_CHUNK16, LD, 0, CL>;
+  auto kernel = lba_contract_packed_kernel<BM, BN, TM, TN, PQ, false, ORD_CHUNK16, LD, 0, CL, H16>;
   constexpr size_t smem = packed_cluster_smem_bytes<BM, BN, TM, TN>();
   static_assert(smem <= 48 * 1024, "no opt-in needed");
   cudaLaunchConfig_t cfg = {};
@@ -29,16 +29,18 @@ cudaError_t launch(const Problem& p, cudaStream_t stream) {
 
 template <int PQ>
 cudaError_t by_loader(int load, const Problem& p, cudaStream_t stream) {
+  // an accumulator value with at most 7 mantissa bits (low 16 bits of the binary32 pattern clear) is a bfloat16
+  const bool h16 = (p.qa.mask & 0xFFFFu) == 0u;
   switch (load) {
-    case LD_GEMM_VEC: return launch<PQ, LD_GEMM_VEC>(p, stream);
-    case LD_CONV_VEC: return launch<PQ, LD_CONV_VEC>(p, stream);
+    case LD_GEMM_VEC: return h16 ? launch<PQ, LD_GEMM_VEC, true>(p, stream) : launch<PQ, LD_GEMM_VEC, false>(p, stream);
+    case LD_CONV_VEC: return h16 ? launch<PQ, LD_CONV_VEC, true>(p, stream) : launch<PQ, LD_CONV_VEC, false>(p, stream);
     default: return cudaErrorInvalidValue;  // the byte-wise loader keeps the single-CTA tiles
   }
 }
 
 }  // namespace
 
-// pq: PackedProd.  The caller has checked: floor rounding, chunk-16 order, M_acc <= 7, 16-byte loader.
+// pq: PackedProd.  The caller has checked: floor rounding, chunk-16 order, 16-byte loader.
 cudaError_t launch_cluster_pair(int pq, int load, const Problem& p, cudaStream_t stream) {
   switch (pq) {
     case PQ_NONE: return by_loader<PQ_NONE>(load, p, stream);

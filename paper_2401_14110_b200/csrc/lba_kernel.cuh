@@ -801,14 +801,15 @@ enum PackedProd { PQ_NONE = 0, PQ_MASK = 1, PQ_MASK_SAT = 2 };
 // Bits that must outlive a slab wait in shared memory (per thread: 16 words for the low half of a mask1
 // word, 32 words for the mask2 word in progress), so the common path keeps the forward kernel's registers.
 //
-// CL = 2 (floor, chunk-16 order, accumulator mantissa of at most 7 bits): two CTAs of a thread-block cluster share
+// CL = 2 (floor, chunk-16 order): two CTAs of a thread-block cluster share
 // one output tile.  The chunk sums C_j of the first hierarchy do not depend on each other; only the folds
 // T <- Q_acc(C_j + T), one addition in sixteen, are sequential.  CTA r forms the chunk sums of the chunks j = r, r + 2,
 // ... for the whole tile and folds, in chunk order, all chunks for the column half r of every thread's micro-tile;
-// the chunk sums of the other half cross to the other CTA through distributed shared memory (as bfloat16 pairs: a
-// value with M <= 7 mantissa bits is one exactly), double buffered, with one cluster barrier per pair of chunks.
+// the chunk sums of the other half cross to the other CTA through distributed shared memory, double buffered, with
+// one cluster barrier per pair of chunks.  H16: the chunk sums travel as bfloat16 pairs, which a value with at most 7
+// mantissa bits is exactly (half the traffic, 2 % faster); otherwise as binary32 words.
 // This doubles the CTAs of a small problem without splitting any sequential chain, and both CTAs do the same work.
-template <int BM, int BN, int TM, int TN, int PQ, bool RNE, int ORD, int LD, int STE = 0, int CL = 1>
+template <int BM, int BN, int TM, int TN, int PQ, bool RNE, int ORD, int LD, int STE = 0, int CL = 1, bool H16 = false>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN),
                                   ((TM * TN == 64 && ORD != ORD_CHUNK_SLAB && !RNE) ||
                                    ((LD == LD_ANY || STE != 0) && !RNE && ORD != ORD_CHUNK_SLAB))
@@ -854,7 +855,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
   const int64_t m0 = (int64_t)(blockIdx.x / CL) * BM;
   const int64_t n0 = (int64_t)blockIdx.y * BN;
   const int nslab = (int)((p.K + BK - 1) / BK);
-  // CL = 2: chunk sums in flight from CTA 1 to CTA 0, [buffer][group of 4 pairs][thread] as uint4 of bfloat16 pairs
+  // CL = 2: chunk sums in flight between the two CTAs, [buffer][group of 2 pairs][thread] as uint4
   uint4* const hand = reinterpret_cast<uint4*>(reinterpret_cast<uint32_t*>(nrm) + 8);
 
   RowLoader<BM, BN, NT, LD> loader;
@@ -1269,7 +1270,11 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
       for (int i = 0; i < TM; ++i)
 #pragma unroll
         for (int j = 0; j < HP; ++j) {
-          const u64 c = recv ? pack2u(recv[i * HP + j] << 16, recv[i * HP + j] & 0xFFFF0000u) : acc1[i][H * HP + j];
+          u64 c = acc1[i][H * HP + j];
+          if (recv) {
+            c = H16 ? pack2u(recv[i * HP + j] << 16, recv[i * HP + j] & 0xFFFF0000u)
+                    : pack2u(recv[2 * (i * HP + j)], recv[2 * (i * HP + j) + 1]);
+          }
           float lo, hi;
           unpack2(add2_rz_ftz(c, T[i][j]), lo, hi);
           lo = and_bits(lo, mask);
@@ -1294,30 +1299,40 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
       }
     };
     auto fold_received = [&](auto half_tag, int q) {
-      uint32_t w[TM * HP];
+      constexpr int NG = H16 ? TM * HP / 4 : TM * HP / 2;  // 16-byte groups per thread and chunk
+      uint32_t w[4 * NG];
 #pragma unroll
-      for (int g = 0; g < TM * HP / 4; ++g) {
-        const uint4 v = hand[((q & 1) * (TM * HP / 4) + g) * NT + tid];
+      for (int g = 0; g < NG; ++g) {
+        const uint4 v = hand[((q & 1) * NG + g) * NT + tid];
         w[g * 4 + 0] = v.x; w[g * 4 + 1] = v.y; w[g * 4 + 2] = v.z; w[g * 4 + 3] = v.w;
       }
       u2 = fold(half_tag, std::true_type(), w) * p.inv_top;
     };
-    // chunk sums of the column half `other` as bfloat16 pairs (exact for M <= 7) into the other CTA's buffer
+    // chunk sums of the column half `other` into the other CTA's buffer, 16 bytes per store
     auto send = [&](auto other_tag, int q) {
       constexpr int O = decltype(other_tag)::value;
+      if constexpr (H16) {
 #pragma unroll
-      for (int g = 0; g < TM * HP / 4; ++g) {
-        uint32_t w[4];
+        for (int g = 0; g < TM * HP / 4; ++g) {
+          uint32_t w[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int idx = g * 4 + e;
-          float lo, hi;
-          unpack2(acc1[idx / HP][O * HP + idx % HP], lo, hi);
-          w[e] = (__float_as_uint(lo) >> 16) | (__float_as_uint(hi) & 0xFFFF0000u);
+          for (int e = 0; e < 4; ++e) {
+            const int idx = g * 4 + e;
+            float lo, hi;
+            unpack2(acc1[idx / HP][O * HP + idx % HP], lo, hi);
+            w[e] = (__float_as_uint(lo) >> 16) | (__float_as_uint(hi) & 0xFFFF0000u);
+          }
+          const uint32_t dst = hand_remote + (uint32_t)(((q & 1) * (TM * HP / 4) + g) * NT + tid) * 16u;
+          asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                       "r"(w[3]) : "memory");
         }
-        const uint32_t dst = hand_remote + (uint32_t)(((q & 1) * (TM * HP / 4) + g) * NT + tid) * 16u;
-        asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
-                     "r"(w[3]) : "memory");
+      } else {
+#pragma unroll
+        for (int g = 0; g < TM * HP / 2; ++g) {
+          const u64 c0 = acc1[(2 * g) / HP][O * HP + (2 * g) % HP], c1 = acc1[(2 * g + 1) / HP][O * HP + (2 * g + 1) % HP];
+          const uint32_t dst = hand_remote + (uint32_t)(((q & 1) * (TM * HP / 2) + g) * NT + tid) * 16u;
+          asm volatile("st.shared::cluster.v2.u64 [%0], {%1, %2};" ::"r"(dst), "l"(c0), "l"(c1) : "memory");
+        }
       }
     };
 
@@ -1523,10 +1538,10 @@ template <int BM, int BN>
 constexpr size_t packed_smem_bytes() {
   return sizeof(float2) * 2 * BK * BM + sizeof(float) * 2 * BK * BN + sizeof(unsigned) * 8;
 }
-// the cluster variant adds the double-buffered hand-over of chunk sums (one bfloat16 per output of a column half and buffer)
+// the cluster variant adds the double-buffered hand-over of chunk sums (one word per output of a column half and buffer)
 template <int BM, int BN, int TM, int TN>
 constexpr size_t packed_cluster_smem_bytes() {
-  return packed_smem_bytes<BM, BN>() + sizeof(uint32_t) * 2 * (BM / TM) * (BN / TN) * (TM * (TN / 4));
+  return packed_smem_bytes<BM, BN>() + sizeof(uint32_t) * 2 * (BM / TM) * (BN / TN) * (TM * (TN / 2));
 }
 // the mask variant adds its two per-thread stashes (16 + 32 words for the 4x8 micro-tile)
 template <int BM, int BN, int TM, int TN>
@@ -1542,7 +1557,7 @@ constexpr size_t packed_ste_smem_bytes() {
 struct TileInfo { int bm, bn, tm, tn; };
 constexpr int TILE_COUNT = 4;
 constexpr int TILE_UMMA = 4;  // override value that selects the tensor-core-product kernel (128 x 64 tile)
-constexpr int TILE_PAIR = 5;  // 64x64 tile shared by a cluster of two CTAs (chunk-16 order, floor, M_acc <= 7)
+constexpr int TILE_PAIR = 5;  // 64x64 tile shared by a cluster of two CTAs (chunk-16 order, floor rounding)
 __host__ inline TileInfo tile_info(int t) {
   const TileInfo tab[TILE_COUNT] = {{128, 128, 8, 8}, {128, 64, 4, 8}, {64, 64, 4, 8}, {32, 32, 4, 4}};
   return tab[t];

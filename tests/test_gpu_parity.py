@@ -467,7 +467,7 @@ def test_fixed_point_conv_batched_and_errors():
         lba.lba_gemm_ste_mask(a2, b2, prod, acc, SEQ, 1, lba.STE_OF)
 
 
-@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_paper", "m4e4", "m4e3_mnist", "m7e4_no_uf"])
+@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_paper", "m4e4", "m10e5", "mixed", "m4e3_mnist", "m7e4_no_uf"])
 def test_cluster_pair_tile_is_exact(name):
     # two CTAs per output tile, each taking every second chunk of 16 (tile override 5): same bits as the oracle
     prod, acc = FORMATS[name]
@@ -491,12 +491,12 @@ def test_cluster_pair_tile_is_exact(name):
             got = lba.lba_conv2d(x.to(DEV), wt.to(DEV), one.to(DEV), one.to(DEV), None, stride, pad, prod, acc, CHK, 16)
             want = orc.conv2d(x.numpy(), wt.numpy(), 1.0, 1.0, None, stride, pad, prod.as_tuple(), acc.as_tuple(), CHK, 16)
             assert_bit_equal(got, want, f"pair tile {name} conv {case}")
-        # not eligible: falls back to the automatic choice, still exact
-        p10, a10 = FORMATS["m10e5"]
+        # not eligible (nearest-even): falls back to the automatic choice, still exact
+        pr, ar = FORMATS["m7e4_code_rne"]
         A, B = _overflow_case(40, 40, 64, 3, 5)
         one = torch.ones(1)
-        assert "pair" not in lba.describe_plan(40, 40, 64, p10, a10, CHK, 16)
-        assert_bit_equal(gpu_gemm(A, B, one, one, None, p10, a10, CHK, 16), ref_gemm(A, B, one, one, None, p10, a10, CHK, 16))
+        assert "pair" not in lba.describe_plan(40, 40, 64, pr, ar, CHK, 16)
+        assert_bit_equal(gpu_gemm(A, B, one, one, None, pr, ar, CHK, 16), ref_gemm(A, B, one, one, None, pr, ar, CHK, 16))
     finally:
         lba.set_tile_override(-1)
     assert lba.device_error() == 0
