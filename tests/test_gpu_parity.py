@@ -491,6 +491,20 @@ def test_cluster_pair_tile_is_exact(name):
             got = lba.lba_conv2d(x.to(DEV), wt.to(DEV), one.to(DEV), one.to(DEV), None, stride, pad, prod, acc, CHK, 16)
             want = orc.conv2d(x.numpy(), wt.numpy(), 1.0, 1.0, None, stride, pad, prod.as_tuple(), acc.as_tuple(), CHK, 16)
             assert_bit_equal(got, want, f"pair tile {name} conv {case}")
+        # batched problems (the grid's third dimension), per-row scales and a bias; K = 0
+        Ab = synth.random_codes((3, 70, 96), 71).to(DEV)
+        Bb = synth.random_codes((3, 45, 96), 72).to(DEV)
+        sa_rows = (torch.rand(70, generator=torch.Generator().manual_seed(1)) + 0.5).to(DEV)
+        sb_cols = (torch.rand(45, generator=torch.Generator().manual_seed(2)) + 0.5).to(DEV)
+        bias = torch.randn(45, generator=torch.Generator().manual_seed(3)).to(DEV)
+        gb = lba.lba_gemm_batched(Ab, Bb, sa_rows, sb_cols, bias, prod, acc, CHK, 16)
+        for z in range(3):
+            want = orc.gemm(Ab[z].cpu().numpy(), Bb[z].cpu().numpy(), sa_rows.cpu().numpy(), sb_cols.cpu().numpy(),
+                            bias.cpu().numpy(), prod.as_tuple(), acc.as_tuple(), CHK, 16)
+            assert_bit_equal(gb[z], want, f"pair tile {name} batched problem {z}")
+        empty = lba.lba_gemm(torch.empty((5, 0), dtype=torch.uint8, device=DEV), torch.empty((7, 0), dtype=torch.uint8, device=DEV),
+                             torch.ones(1, device=DEV), torch.ones(1, device=DEV), None, prod, acc, CHK, 16)
+        assert empty.shape == (5, 7) and (empty == 0).all()
         # not eligible (nearest-even): falls back to the automatic choice, still exact
         pr, ar = FORMATS["m7e4_code_rne"]
         A, B = _overflow_case(40, 40, 64, 3, 5)
