@@ -516,6 +516,48 @@ def test_cluster_pair_tile_is_exact(name):
     assert lba.device_error() == 0
 
 
+def test_random_shapes_pair_tile_masks_and_fixed_point():
+    # seeded random shapes, data regimes and formats through the cluster-pair tile, both mask kernels and the
+    # fixed-point kernel: every output bit against the oracle
+    rng = np.random.default_rng(2024)
+    floats = [FORMATS[n] for n in ("m7e4_code", "m7e4_paper", "m4e4", "m10e5", "m4e3_mnist", "m7e4_no_uf", "m5e6")]
+    for it in range(48):
+        M, N = int(rng.integers(1, 200)), int(rng.integers(1, 200))
+        K = int(rng.integers(1, 40)) * 16 if it % 3 else int(rng.integers(1, 700))
+        regime = int(rng.integers(0, 3))
+        if regime == 2:
+            A, _, B, _ = synth.gemm_case(M, N, K, config=300 + it)
+        else:
+            A, B = synth.random_codes((M, K), 1000 + it), synth.random_codes((N, K), 5000 + it)
+            if regime == 1:
+                A, B = A & 0x7F, B & 0x7F
+        pf, af = floats[it % len(floats)]
+        sa, sb = torch.tensor([0.7]), torch.rand(N, generator=torch.Generator().manual_seed(it)) + 0.5
+        what = f"case {it}: {M}x{N}x{K} regime {regime}"
+        lba.set_tile_override(5)
+        try:
+            got = gpu_gemm(A, B, sa, sb, None, pf, af, CHK, 16)
+        finally:
+            lba.set_tile_override(-1)
+        assert_bit_equal(got, ref_gemm(A, B, sa, sb, None, pf, af, CHK, 16), what + " pair tile")
+        for order, chunk in ((SEQ, 1), (CHK, 16)):
+            kinds = [(lba.STE_OF, orc.STE_OF, 0.0, 0.0)] + ([(lba.STE_DIFF, orc.STE_DIFF, 2.0 ** -18, 0.3)] if it % 2 == 0 else [])
+            for kind, okind, e1, e2 in kinds:
+                g1, g2 = lba.lba_gemm_ste_mask(A.to(DEV), B.to(DEV), pf, af, order, chunk, kind, e1, e2)
+                w1, w2 = orc.gemm_ste_mask(A.numpy(), B.numpy(), pf.as_tuple(), af.as_tuple(), order, chunk, okind, e1, e2)
+                assert (_u32(g1) == w1).all(), what + f" mask1 order {order} kind {kind}"
+                assert w2 is None or (_u32(g2) == w2).all(), what + f" mask2 order {order} kind {kind}"
+        bp, ba = int(rng.integers(-8, 8)), int(rng.integers(-10, 8))
+        Bp, Ba = int(rng.integers(6, 25)), int(rng.integers(6, 25))
+        if ba - bp > 0 and (Bp - 1) + (ba - bp) > 30:
+            continue
+        fp, fa = fixed_point_format(Bp, bp, bool(it % 2)), fixed_point_format(Ba, ba, bool(it % 2))
+        order, chunk = [(SEQ, 1), (CHK, 16), (CHK, 7), (CHK, 48)][it % 4]
+        assert_bit_equal(gpu_gemm(A, B, sa, sb, None, fp, fa, order, chunk), ref_gemm(A, B, sa, sb, None, fp, fa, order, chunk),
+                         what + f" fixed point {fp.as_tuple()} {fa.as_tuple()} order {order} chunk {chunk}")
+    assert lba.device_error() == 0
+
+
 def test_zero_and_empty_shapes():
     prod, acc = code_domain_formats(7, 4)
     one = torch.ones(1)
