@@ -26,7 +26,8 @@
  *                         The last chunk may be short.
  *
  * All device pointers must belong to the current CUDA device.  The library allocates no
- * memory, keeps no state between calls except the last CUDA error code, and never
+ * memory, keeps no state between calls except the last CUDA error code (and the testing hook
+ * lba_set_tile_override), and never
  * synchronises: work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default
  * stream).  Format structs are read on the host during the call.
  *
@@ -164,7 +165,9 @@ int lba_conv2d(const uint8_t* x, const uint8_t* w, const float* scale_x, int sca
  * the caller's device workspace, the kernel runs, and `out` (host) receives the result; all
  * of it is enqueued on `stream`, so the caller synchronises the stream before reading `out`.
  * `workspace` is device memory, 256-byte aligned, of at least lba_*_host_workspace_bytes(...)
- * bytes; the library does not allocate. */
+ * bytes; the library does not allocate.  A shape whose operand or output byte counts do not fit
+ * in 62 bits is refused (the size functions return 0, the calls LBA_ERR_SHAPE) before anything
+ * is copied. */
 size_t lba_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int scale_a_len, int scale_b_len,
                                      int has_bias);
 int lba_gemm_host(const uint8_t* A, const uint8_t* B, const float* scale_a, int scale_a_len, const float* scale_b,
@@ -213,26 +216,23 @@ int lba_gemm_host_static(const uint8_t* A, const uint8_t* B, const float* scale_
 int lba_count_nan_codes(const uint8_t* codes, int64_t n, unsigned long long* count, void* stream);
 
 /* Which kernel variant a call with these arguments would run, as text, e.g.
- * "tile=64x64x16 micro=4x8 q=floor_fast order=chunk16 load=gemm_vec grid=128x128".
+ * "tile=64x64x16 micro=4x8 q=floor_fast pq=none kernel=packed order=chunk16 load=gemm_vec grid=128x128"
+ * (pq: what Q_prod does beyond its flush -- none, cut = mantissa cut, cut_sat = cut and saturation; kernel: the
+ * packed two-outputs-per-instruction kernel or the generic scalar one).
  * is_conv selects the loader family; for a convolution pass M = B*H_out*W_out, N = C_out,
  * K = KH*KW*C_in and vec_ok = (C_in % 16 == 0 and pointers aligned).  Returns LBA_OK or the
  * error the real call would return; buf may be NULL. */
 int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, const lba_fmt* acc_fmt, int order,
                       int chunk, int is_conv, int vec_ok, char* buf, size_t buf_len);
 
-/* Testing and tuning hook: force the CTA tile (0 = 128x128, 1 = 128x64, 2 = 64x64, 3 = 32x32
- * outputs; 4 = the experimental kernel whose products come from the tensor cores, 128x64 outputs, used only
- * for the fast floor quantiser in chunk-16 order and ignored otherwise; 5 = the 64x64 tile shared by a cluster of two
- * CTAs, each taking every second chunk, used only in chunk-16 order with floor rounding and 16-byte loads, ignored
- * otherwise; -1 = automatic choice, the default).  For
- * lba_gemm_ste_mask, 3 selects the scalar tracking kernel where the packed one would run.  Process-wide; results never
- * depend on the tile, only speed does.  Returns LBA_OK, or LBA_ERR_SHAPE for an unknown tile. */
+/* Testing and tuning hook: force the CTA tile (0 = 128x128, 1 = 128x64, 2 = 64x64, 3 = 32x32 outputs; 5 = the 64x64
+ * tile shared by a cluster of two CTAs, each taking every second chunk, used only in chunk-16 order with floor
+ * rounding and 16-byte loads, ignored otherwise; -1 = automatic choice, the default).  For lba_gemm_ste_mask, 3
+ * selects the scalar tracking kernel where the packed one would run.  Results never depend on the tile, only speed
+ * does.  The setting is one process-wide word (an atomic store): it is meant for tests and tuning runs, it applies
+ * to every thread's later calls, and a caller that changes it while other threads are inside the library gets an
+ * unspecified mix of old and new tiles, never a wrong result.  Returns LBA_OK, or LBA_ERR_SHAPE for an unknown tile. */
 int lba_set_tile_override(int tile);
-
-/* Error word of the device code: kernels that wait on hardware barriers bound every wait, and a wait that runs
- * out stores a non-zero code here instead of hanging.  Reads and clears the word; synchronises the device.
- * 0 means no kernel has reported a problem since the last call. */
-int lba_device_error(int* code);
 
 const char* lba_status_string(int status);
 int lba_last_cuda_error(void); /* cudaError_t of the most recent failed CUDA call in this thread, else 0 */

@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "liblba.so")
 
 EXPORTS = ["lba_gemm", "lba_gemm_batched", "lba_gemm_last_overflow", "lba_gemm_ste_mask", "lba_conv2d", "lba_gemm_host_workspace_bytes", "lba_gemm_host",
            "lba_conv2d_host_workspace_bytes", "lba_conv2d_host", "lba_gemm_host_static", "lba_count_nan_codes", "lba_describe_plan",
-           "lba_set_tile_override", "lba_device_error", "lba_status_string", "lba_last_cuda_error", "lba_version"]
+           "lba_set_tile_override", "lba_status_string", "lba_last_cuda_error", "lba_version"]
 
 
 class LbaError(RuntimeError):
@@ -282,16 +282,9 @@ def count_nan_codes(codes, stream=None):
     return int(count.item())
 
 
-def device_error():
-    """Error word of the device code (0 = none since the last call); synchronises."""
-    lib = load_library()
-    code = C.c_int(0)
-    _check(lib.lba_device_error(C.byref(code)))
-    return code.value
-
-
 def set_tile_override(tile):
-    """Force the CTA tile (0..3) or restore the automatic choice (-1).  Speed only; results are unchanged."""
+    """Force the CTA tile (0..3, 5 = cluster pair) or restore the automatic choice (-1).  A testing hook: process-wide.
+    Speed only; results are unchanged."""
     _check(load_library().lba_set_tile_override(int(tile)))
 
 

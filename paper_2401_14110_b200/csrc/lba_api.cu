@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <atomic>
 #include <mutex>
 
 #include "../../include/lba.h"
@@ -20,8 +21,6 @@ LBA_DECL(QM_RNE_FULL, ORD_SEQ) LBA_DECL(QM_RNE_FULL, ORD_CHUNK_SLAB) LBA_DECL(QM
 LBA_DECL(QM_RNE_WIDE, ORD_SEQ) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_SLAB) LBA_DECL(QM_RNE_WIDE, ORD_CHUNK_ANY)
 #undef LBA_DECL
 
-cudaError_t launch_umma_family(int load, const Problem& p, cudaStream_t stream);
-cudaError_t read_umma_error(int* code);
 cudaError_t launch_last_overflow(int qm, int load, const Problem& p, cudaStream_t stream);
 cudaError_t launch_ste_mask(int qm, int ord, int diff, int load, const Problem& p, cudaStream_t stream);
 cudaError_t launch_ste_packed(int pq, int chunk16, int load, const Problem& p, cudaStream_t stream);
@@ -31,7 +30,7 @@ cudaError_t launch_cluster_pair(int pq, int load, const Problem& p, cudaStream_t
 namespace {
 
 thread_local int g_last_cuda_error = 0;
-int g_tile_override = -1;
+std::atomic<int> g_tile_override{-1};  // testing and tuning hook (lba_set_tile_override)
 
 int cuda_fail(cudaError_t e) {
   g_last_cuda_error = (int)e;
@@ -257,19 +256,28 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
   return LBA_OK;
 }
 
+// SM count of the current device, asked once per device (148 if the query fails).
+int sm_count() {
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  int v = cached[dev].load(std::memory_order_relaxed);
+  if (v > 0) return v;
+  if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+  cached[dev].store(v, std::memory_order_relaxed);
+  return v;
+}
+
 // Tile choice.  All CTAs of a launch have the same work and K is never split, so the launch ends when the
 // busiest SM has run its ceil(CTAs / SMs) tiles; larger tiles spend fewer instructions per MAC (eff, measured
 // on B200 with every SM loaded), smaller ones fill the SMs more evenly.  Pick the cheapest by that model.
 // pair_ok: the call qualifies for the 64x64 tile shared by a cluster of two CTAs (TILE_PAIR)
 int choose_tile(int64_t M, int64_t N, int64_t batch, int qm, int ord, int load, bool pair_ok = false) {
   (void)qm;
-  if (g_tile_override >= 0 && g_tile_override < TILE_COUNT) return g_tile_override;
-  if (g_tile_override == TILE_PAIR && pair_ok) return TILE_PAIR;
-  int dev = 0, sms = 148;
-  if (cudaGetDevice(&dev) == cudaSuccess) {
-    int v = 0;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
-  }
+  const int forced = g_tile_override.load(std::memory_order_relaxed);
+  if (forced >= 0 && forced < TILE_COUNT) return forced;
+  if (forced == TILE_PAIR && pair_ok) return TILE_PAIR;
+  const int sms = sm_count();
   // relative MAC rate of each tile with every SM loaded (8192^2 x 1024 and 4096 x 3072 x 768 GEMMs)
   const double eff_seq[TILE_COUNT] = {1.00, 0.91, 0.95, 0.84};
   const double eff_chunk[TILE_COUNT] = {0.97, 0.96, 1.00, 0.89};
@@ -347,13 +355,6 @@ int run(const Problem& p, const Plan& pl, int load, cudaStream_t stream) {
     const cudaError_t e = launch_fixed(pl.ord, load, p, stream);
     return e == cudaSuccess ? LBA_OK : cuda_fail(e);
   }
-  if (g_tile_override == TILE_UMMA) {  // the tensor-core-product kernel, where it applies
-    if (pl.qm == QM_FLOOR_FAST && pl.ord == ORD_CHUNK16) {
-      if ((p.N + 63) / 64 > 65535) return LBA_ERR_SHAPE;
-      const cudaError_t e = launch_umma_family(load, p, stream);
-      return e == cudaSuccess ? LBA_OK : cuda_fail(e);
-    }
-  }
   const bool pair_ok = pl.ord == ORD_CHUNK16 && (pl.qm == QM_FLOOR_FAST || pl.qm == QM_FLOOR_FULL) && load != LD_ANY &&
                        2 * ((p.M + 63) / 64) <= 2147483647LL;
   const int tile = choose_tile(p.M, p.N, p.batch, pl.qm, pl.ord, load, pair_ok);
@@ -396,6 +397,13 @@ __global__ void count_nan_codes_kernel(const uint8_t* codes, int64_t n, unsigned
 
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Sizes of the host-buffer variants are formed in size_t; a shape whose operand or output byte count does not fit
+// well inside 63 bits is refused before any product can wrap.
+bool sizes_fit(double a_bytes, double b_bytes, double out_bytes) {
+  const double limit = 4611686018427387904.0;  // 2^62
+  return a_bytes < limit && b_bytes < limit && out_bytes < limit && a_bytes + b_bytes + out_bytes < limit;
+}
+
 }  // namespace
 }  // namespace lba
 
@@ -405,17 +413,11 @@ extern "C" {
 
 int lba_version(void) { return 1; }
 
-int lba_device_error(int* code) {
-  if (!code) return LBA_ERR_NULL;
-  const cudaError_t e = read_umma_error(code);
-  return e == cudaSuccess ? LBA_OK : cuda_fail(e);
-}
-
 int lba_last_cuda_error(void) { return g_last_cuda_error; }
 
 int lba_set_tile_override(int tile) {
-  if (tile < -1 || tile > TILE_PAIR) return LBA_ERR_SHAPE;
-  g_tile_override = tile;
+  if (tile < -1 || tile > TILE_PAIR || tile == TILE_COUNT) return LBA_ERR_SHAPE;
+  g_tile_override.store(tile, std::memory_order_relaxed);
   return LBA_OK;
 }
 
@@ -588,7 +590,7 @@ int lba_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, 
   const int load = vec ? LD_GEMM_VEC : LD_ANY;
   // the overflow masks in sequential and chunk-16 order come from the packed kernel (tile override 3 keeps the
   // scalar tracking kernel, for tests and comparisons); everything else from the scalar one
-  const bool packed = ste == LBA_STE_OF && (!chunked || chunk == BK) && g_tile_override != 3;
+  const bool packed = ste == LBA_STE_OF && (!chunked || chunk == BK) && g_tile_override.load(std::memory_order_relaxed) != 3;
   const cudaError_t e = packed ? launch_ste_packed(pl.qm == QM_FLOOR_FAST ? PQ_NONE : pl.pq, chunked ? 1 : 0, load, p, (cudaStream_t)stream)
                                : launch_ste_mask(pl.qm, ord, ste == LBA_STE_DIFF, load, p, (cudaStream_t)stream);
   return e == cudaSuccess ? LBA_OK : cuda_fail(e);
@@ -626,6 +628,7 @@ int lba_conv2d(const uint8_t* x, const uint8_t* w, const float* scale_x, int sca
 size_t lba_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int scale_a_len, int scale_b_len,
                                      int has_bias) {
   if (M < 0 || N < 0 || K < 0 || scale_a_len < 0 || scale_b_len < 0) return 0;
+  if (!sizes_fit((double)M * (double)K, (double)N * (double)K, 4.0 * (double)M * (double)N)) return 0;
   size_t b = 0;
   b += round_up((size_t)M * K, 256) + round_up((size_t)N * K, 256);
   b += round_up((size_t)scale_a_len * 4, 256) + round_up((size_t)scale_b_len * 4, 256);
@@ -638,7 +641,8 @@ int lba_gemm_host(const uint8_t* A, const uint8_t* B, const float* scale_a, int 
                   int scale_b_len, const float* bias, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt,
                   const lba_fmt* acc_fmt, int order, int chunk, float* out, void* workspace,
                   size_t workspace_bytes, void* stream) {
-  if (M < 0 || N < 0 || K < 0) return LBA_ERR_SHAPE;
+  if (M < 0 || N < 0 || K < 0 || K > 2147483647LL) return LBA_ERR_SHAPE;
+  if (!sizes_fit((double)M * (double)K, (double)N * (double)K, 4.0 * (double)M * (double)N)) return LBA_ERR_SHAPE;
   if (!scale_a || !scale_b) return LBA_ERR_NULL;
   if (!(scale_a_len == 1 || scale_a_len == M) || !(scale_b_len == 1 || scale_b_len == N)) return LBA_ERR_SCALE_LEN;
   Plan pl;
@@ -674,6 +678,7 @@ size_t lba_conv2d_host_workspace_bytes(int B, int H, int W, int C_in, int C_out,
   ConvGeom g;
   if (conv_geom(B, H, W, C_in, C_out, KH, KW, stride_h, stride_w, pad_h, pad_w, &g) != LBA_OK) return 0;
   if (scale_x_len < 0 || scale_w_len < 0) return 0;
+  if (!sizes_fit((double)B * H * W * C_in, (double)C_out * (double)g.K, 4.0 * (double)g.M * C_out)) return 0;
   size_t b = 0;
   b += round_up((size_t)B * H * W * C_in, 256) + round_up((size_t)C_out * g.K, 256);
   b += round_up((size_t)scale_x_len * 4, 256) + round_up((size_t)scale_w_len * 4, 256);
@@ -690,6 +695,7 @@ int lba_conv2d_host(const uint8_t* x, const uint8_t* w, const float* scale_x, in
   ConvGeom g;
   int st = conv_geom(B, H, W, C_in, C_out, KH, KW, stride_h, stride_w, pad_h, pad_w, &g);
   if (st != LBA_OK) return st;
+  if (!sizes_fit((double)B * H * W * C_in, (double)C_out * (double)g.K, 4.0 * (double)g.M * C_out)) return LBA_ERR_SHAPE;
   if (!x || !w || !out || !scale_x || !scale_w) return LBA_ERR_NULL;
   if (!(scale_x_len == 1 || scale_x_len == g.M) || !(scale_w_len == 1 || scale_w_len == C_out)) return LBA_ERR_SCALE_LEN;
   Plan pl;
@@ -745,17 +751,24 @@ int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, 
   }
   const bool pair_ok = pl.ord == ORD_CHUNK16 && (pl.qm == QM_FLOOR_FAST || pl.qm == QM_FLOOR_FULL) && load != LD_ANY;
   const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, 1, pl.qm, pl.ord, load, pair_ok);
+  // which kernel runs and what Q_prod costs there beyond the flush
+  const bool packed = pl.ord != ORD_CHUNK_ANY &&
+                      (pl.qm == QM_FLOOR_FAST || pl.qm == QM_FLOOR_FULL || (pl.qm == QM_RNE_FULL && pl.rne_packed));
+  const char* const kern = packed ? "packed" : "generic";
+  const char* const pq = pl.qm == QM_FLOOR_FAST || pl.qm == QM_RNE_WIDE ? "none"
+                         : (pl.pq == PQ_MASK_SAT ? "cut_sat" : (pl.pq == PQ_MASK ? "cut" : "none"));
   if (tile == TILE_PAIR) {
     if (buf && buf_len)
-      std::snprintf(buf, buf_len, "tile=64x64x%d pair micro=4x8 q=%s order=%s load=%s grid=%lldx%lld", BK, kQmName[pl.qm],
-                    kOrdName[pl.ord], kLdName[load], (long long)(2 * ((M + 63) / 64)), (long long)((N + 63) / 64));
+      std::snprintf(buf, buf_len, "tile=64x64x%d pair micro=4x8 q=%s pq=%s kernel=%s order=%s load=%s grid=%lldx%lld", BK,
+                    kQmName[pl.qm], pq, kern, kOrdName[pl.ord], kLdName[load], (long long)(2 * ((M + 63) / 64)),
+                    (long long)((N + 63) / 64));
     return LBA_OK;
   }
   const TileInfo ti = tile_info(tile);
   if (buf && buf_len)
-    std::snprintf(buf, buf_len, "tile=%dx%dx%d micro=%dx%d q=%s order=%s load=%s grid=%lldx%lld", ti.bm, ti.bn, BK,
-                  ti.tm, ti.tn, kQmName[pl.qm], kOrdName[pl.ord], kLdName[load], (long long)((M + ti.bm - 1) / ti.bm),
-                  (long long)((N + ti.bn - 1) / ti.bn));
+    std::snprintf(buf, buf_len, "tile=%dx%dx%d micro=%dx%d q=%s pq=%s kernel=%s order=%s load=%s grid=%lldx%lld", ti.bm, ti.bn,
+                  BK, ti.tm, ti.tn, kQmName[pl.qm], pq, kern, kOrdName[pl.ord], kLdName[load],
+                  (long long)((M + ti.bm - 1) / ti.bm), (long long)((N + ti.bn - 1) / ti.bn));
   return LBA_OK;
 }
 

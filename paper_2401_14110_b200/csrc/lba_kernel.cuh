@@ -1556,7 +1556,6 @@ constexpr size_t packed_ste_smem_bytes() {
 // 64 or 128 threads, 4x8 in 32x64, 32x128, 64x128, 128x128, 64x256 tiles, a one-warp 32x32 tile.
 struct TileInfo { int bm, bn, tm, tn; };
 constexpr int TILE_COUNT = 4;
-constexpr int TILE_UMMA = 4;  // override value that selects the tensor-core-product kernel (128 x 64 tile)
 constexpr int TILE_PAIR = 5;  // 64x64 tile shared by a cluster of two CTAs (chunk-16 order, floor rounding)
 __host__ inline TileInfo tile_info(int t) {
   const TileInfo tab[TILE_COUNT] = {{128, 128, 8, 8}, {128, 64, 4, 8}, {64, 64, 4, 8}, {32, 32, 4, 4}};

@@ -74,3 +74,25 @@ def test_host_side_checks_run_before_any_cuda_call():
                           C.byref(af), 0, 16, fake, None) == -2
     assert lib.lba_gemm_host_workspace_bytes(4, 4, 16, 1, 1, 0) == 256 * 5
     assert lib.lba_set_tile_override(9) == -2 and lib.lba_set_tile_override(-1) == 0
+
+
+def test_host_variants_refuse_shapes_whose_byte_counts_would_wrap():
+    # M*K, N*K and 4*M*N are formed in size_t inside the host-buffer variants: a shape for which one of them does
+    # not fit must come back as an error code (and a workspace size of 0), never as a small wrapped size
+    lib = lba.load_library()
+    p, a = code_domain_formats(7, 4)
+    pf, af = lba._fmt(p), lba._fmt(a)
+    fake = C.c_void_p(256)
+    huge = 1 << 62
+    assert lib.lba_gemm_host_workspace_bytes(huge, 1, 4, 1, 1, 0) == 0          # M*K = 2^64
+    assert lib.lba_gemm_host_workspace_bytes(1 << 31, 1 << 31, 16, 1, 1, 0) == 0  # 4*M*N = 2^64
+    assert lib.lba_gemm_host_workspace_bytes(1 << 20, 1 << 20, 16, 1, 1, 0) > 0   # 4 TiB: large, but it fits
+    for (M, N, K) in ((huge, 1, 4), (1 << 31, 1 << 31, 16), (4, 4, 1 << 31)):
+        assert lib.lba_gemm_host(fake, fake, fake, 1, fake, 1, None, M, N, K, C.byref(pf), C.byref(af), 1, 16, fake, fake,
+                                 C.c_size_t(1 << 40), None) == -2
+        assert lib.lba_gemm_host_static(fake, fake, fake, 1, fake, 1, None, M, N, K, C.byref(pf), C.byref(af), 1, 16, fake,
+                                        None) in (-2, -8)
+    # convolution: B*H*W*C_in beyond int32 is refused by the geometry check already; the output count is guarded too
+    assert lib.lba_conv2d_host_workspace_bytes(1 << 20, 1, 1, 1, 1 << 20, 1, 1, 1, 1, 0, 0, 1, 1, 0) > 0
+    assert lib.lba_conv2d_host_workspace_bytes(1 << 30, 1, 1, 1, 1 << 30, 1, 1, 1, 1, 0, 0, 1, 1, 0) == 0     # 4*M*C_out = 2^62
+    assert lib.lba_conv2d_host_workspace_bytes(1 << 30, 2, 2, 1, 1, 1, 1, 1, 1, 0, 0, 1, 1, 0) == 0
