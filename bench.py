@@ -100,8 +100,16 @@ def mode_of(desc: str, ste=None, fixed=False) -> str:
 
 
 def peak_gmacs(mode, chunk, sm_count, mhz):
+    """(ALU-issue roofline in GMAC/s, issue slots per MAC of the minimal mix, tighter pipe limit or None).
+
+    The roofline every fraction is quoted against is the issue roofline: lanes issued per clock x clock / issue slots
+    per emulated MAC of the minimal mix.  Where one pipe alone needs more clocks than the issue slots (the logic pipe
+    holds every instruction for two clocks), that tighter limit is reported beside it, not used as the denominator."""
+    slots = min_issue_slots(mode, chunk)
     clk, which = clocks_per_warp_mac(mode, chunk)
-    return sm_count * LANES_PER_SM_CLK * mhz * 1e6 / clk / 1e9, clk, which
+    pipe = None if which == "issue" or clk <= slots else {"limit": which, "clocks_per_warp_mac": clk,
+                                                           "peak": sm_count * LANES_PER_SM_CLK * mhz * 1e6 / clk / 1e9}
+    return sm_count * LANES_PER_SM_CLK * mhz * 1e6 / slots / 1e9, slots, pipe
 
 
 # DRAM bytes (read + write) of ONE launch of the dominant kernel, from the ncu captures summarised under profiles/
@@ -377,8 +385,8 @@ def kernel_table(wl, per_call_ms, sm_count, max_mhz):
         e["launches"] += 1
     for key, e in table.items():
         mode = mode_of(key, ste=wl.ste if wl.ste == "diff" else None, fixed=wl.fixed is not None)
-        peak, clk, which = peak_gmacs(mode, wl.chunk if wl.order == 1 else 0, sm_count, max_mhz)
-        e.update(gmacs=e["macs"] / (e["ms"] * 1e-3) / 1e9, mode=mode, peak=peak, clk=clk, limit=which)
+        peak, slots, pipe = peak_gmacs(mode, wl.chunk if wl.order == 1 else 0, sm_count, max_mhz)
+        e.update(gmacs=e["macs"] / (e["ms"] * 1e-3) / 1e9, mode=mode, peak=peak, slots=slots, pipe=pipe)
         e["frac"] = e["gmacs"] / peak
     return table
 
@@ -439,10 +447,10 @@ def other_configs(device, sm_count, max_mhz, headline_wl):
                 table = kernel_table(wl, per, sm_count, max_mhz)
                 (key, e), = table.items()
                 points[wl.name] = {"ms": per[0], "gmacs": e["gmacs"], "mode": e["mode"], "frac": e["frac"]}
-                by_mode.setdefault(e["mode"], []).append((e["gmacs"], e["frac"], e["peak"], key))
+                by_mode.setdefault(e["mode"], []).append((e["gmacs"], e["frac"], e["peak"], key, e["pipe"]))
     modes = {m: {"points": len(v), "gmacs_min": min(x[0] for x in v), "gmacs_median": statistics.median(x[0] for x in v),
                  "gmacs_max": max(x[0] for x in v), "frac_median": statistics.median(x[1] for x in v), "peak": v[0][2],
-                 "mix": MIX[m][4], "kernel": v[0][3]} for m, v in by_mode.items()}
+                 "mix": MIX[m][4], "kernel": v[0][3], "pipe_limit": v[0][4]} for m, v in by_mode.items()}
     out["config5_format_sweep_gemm_8192x8192x8192_chunk16"] = {
         "points": points, "modes": modes, "note": "one warm-up and two timed launches per point; biases by the flex-bias rule "
         "applied to products (b_prod = 2^E - 18, b_acc = b_prod - 2)"}
@@ -639,8 +647,10 @@ def main(argv=None):
         "kernel": dom_key, "kernel_launches_per_step": dom["launches"], "kernel_ms_per_step": dom["ms"],
         "kernel_share_of_step": dom["ms"] / sum(per_call_ms),
         "peak_derivation": f"{sm_count} SMs x {LANES_PER_SM_CLK} lanes issued per clock x {max_mhz:.0f} MHz (clocks.max.sm) / "
-                           f"{dom['clk']:g} clocks per warp-MAC per scheduler, the {dom['limit']} limit of the minimal mix "
-                           f"({MIX[dom['mode']][4]}" + (", plus the fold of every chunk of 16" if wl.order == 1 else "") + ")",
+                           f"{dom['slots']:g} issue slots per emulated MAC of the minimal mix ({MIX[dom['mode']][4]}"
+                           + (f", plus {FOLD.get('rne' if dom['mode'].startswith('rne') else 'floor', FOLD['generic'])[0]:g} per output "
+                              f"per chunk of {wl.chunk}" if wl.order == 1 else "") + ")",
+        "pipe_limit": dom["pipe"],
         "frac_at_sampled_clock": dom["gmacs"] / (dom["peak"] * mhz / max_mhz),
         "whole_step_frac_of_peak": ideal_ms / sum(per_call_ms),
     }

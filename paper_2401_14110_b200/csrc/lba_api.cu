@@ -58,11 +58,13 @@ const char* const kLdName[LD_COUNT] = {"gemm_vec", "conv_vec", "any"};
 constexpr double kMaxProduct = 448.0 * 448.0;  // 200704
 constexpr double kPairEff = 0.91;              // MAC rate of the cluster-pair tile relative to the plain 64x64 tile (measured)
 constexpr int kMinProductExp = -18;            // every product, hence every sum, is a multiple of 2^-18
+constexpr int kProductBits = 8;                // significant bits of a product of two E4M3 values, at most
 
 struct Plan {
   int qm, ord;
   float dec_a, dec_b, c, un1, un2;
   float pk_a, pk_b, nrm_scale, inv_top;
+  float clamp_lim, slab_factor, fold_factor;
   int pq, rne_packed;
   float rne_k_acc, rne_k_prod;
   QConst qp, qa;
@@ -228,17 +230,41 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
     }
   }
 
-  // ---- packed kernel: what Q_prod does beyond the flush; nearest-even rounds on the FP32 pipe by adding
-  // 1.5 * 2^(23-M) * 2^e, which needs that much exponent headroom above the largest carried magnitude
+  // clamp elision (see Problem::clamp_lim): floor never raises a magnitude; nearest-even raises it by at most half a
+  // grid step per rounding, i.e. by the factor 1 + 2^-(M+1): sixteen accumulator roundings and the product's own in a
+  // slab, one in a fold.  A sum at or below R_OF = 2^(e_max+1) (1 - 2^-(M+1)) rounds to at most R_OF.
+  if (nearest) {
+    const double ea = 1.0 + std::ldexp(1.0, -af->man_bits - 1), ep = p_round ? 1.0 + std::ldexp(1.0, -pf->man_bits - 1) : 1.0;
+    pl->clamp_lim = (float)(0.999 * (1.0 - std::ldexp(1.0, -af->man_bits - 1)));
+    pl->slab_factor = (float)(std::pow(ea, 16) * ep * 1.0001);
+    pl->fold_factor = (float)(ea * 1.0001);
+  } else {
+    pl->clamp_lim = 0.999f;
+    pl->slab_factor = 1.0f;
+    pl->fold_factor = 1.0f;
+  }
+
+  // ---- packed kernel: what Q_prod does beyond the flush.  Nearest-even rounds on the FP32 pipe by adding and
+  // subtracting 1.5 * 2^(23-M) * 2^e, which needs that much exponent headroom above the largest carried magnitude.
+  // Its sum is one FMA rounded to nearest, which equals one rounding of the exact sum only under these conditions:
+  //   * the quantised product has no more significant bits than the accumulator (else a product that is the larger
+  //     operand can sit exactly on a tie of the accumulator's grid, which a far smaller sum must break);
+  //   * M_acc <= 10, so that an operand small enough to be lost in the binary32 rounding (below 2^-12 of the larger
+  //     one) is also too small to move the larger one, which lies on the grid, as far as the nearest tie;
+  //   * the product carrier is not scaled down by more than 2^12 on its way into the sum, so that every sum below
+  //     R_UF_acc is a subnormal binary32 number exactly and `.ftz` flushes it (a smaller term could be rounded
+  //     away next to -R_UF_acc and leave R_UF_acc itself standing).
+  // Everything else in nearest-even mode runs in the generic kernel (round-to-odd, then the cut).
   pl->pq = p_sat ? PQ_MASK_SAT : (p_round ? PQ_MASK : PQ_NONE);
-  pl->rne_k_acc = (float)std::ldexp(1.5, 23 - af->man_bits);
-  pl->rne_k_prod = (float)std::ldexp(1.5, 23 - pf->man_bits);
+  pl->rne_k_acc = (float)std::ldexp(1.0, 23 - af->man_bits);
+  pl->rne_k_prod = (float)std::ldexp(1.0, 23 - pf->man_bits);
   pl->rne_packed = 0;
   if (pl->qm == QM_RNE_FULL) {
     const int top_acc = (a_sat ? a_emax + 1 : (int)std::ceil(std::log2(max_sum)) + 1) + ka;
     const int top_prod = 18 + kp;
-    pl->rne_packed = (top_acc + 25 - af->man_bits <= 127) && (top_prod + 25 - pf->man_bits <= 127) &&
-                     af->man_bits <= 21 && pf->man_bits <= 21;
+    const int prod_bits = pf->man_bits + 1 < kProductBits ? pf->man_bits + 1 : kProductBits;
+    pl->rne_packed = (top_acc + 25 - af->man_bits <= 127) && (top_prod + 25 - pf->man_bits <= 127) && af->man_bits <= 10 &&
+                     prod_bits <= af->man_bits + 1 && ka - kp >= -12 && ka - kp <= 60;
   }
 
   // ---- order mode
@@ -334,6 +360,9 @@ void apply_plan(Problem* p, const Plan& pl) {
   p->pk_b = pl.pk_b;
   p->nrm_scale = pl.nrm_scale;
   p->inv_top = pl.inv_top;
+  p->clamp_lim = pl.clamp_lim;
+  p->slab_factor = pl.slab_factor;
+  p->fold_factor = pl.fold_factor;
   p->pq = pl.pq;
   p->rne_packed = pl.rne_packed;
   p->rne_k_acc = pl.rne_k_acc;

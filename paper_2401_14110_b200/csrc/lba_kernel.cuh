@@ -74,7 +74,12 @@ struct Problem {
   float inv_top;       // accumulator carrier -> fraction of 2^(e_max_acc + 1)
   int pq;              // PackedProd: what Q_prod does beyond the flush
   int rne_packed;      // nearest-even: 1 if the packed kernel's exponent headroom suffices
-  float rne_k_acc, rne_k_prod;  // 1.5 * 2^(23 - M) for the accumulator and the product format
+  float rne_k_acc, rne_k_prod;  // 2^(23 - M) for the accumulator and the product format
+  // clamp elision: a slab or fold runs without the magnitude clamp while (bound + growth) * factor < clamp_lim.
+  // Floor never raises a magnitude: factors 1, limit just under 1 (of 2^(e_max+1)).  Nearest-even can raise one by
+  // half a grid step per rounding: slab_factor bounds sixteen such steps (and the product's own rounding),
+  // fold_factor one, and the limit keeps every sum at or below R_OF, which then rounds to at most R_OF.
+  float clamp_lim, slab_factor, fold_factor;
   // straight-through-estimator masks (tracking variants of the scalar kernel only)
   uint32_t *mask1, *mask2;
   int64_t mask2_words;  // ceil(chunks / 32)
@@ -677,16 +682,6 @@ __device__ __forceinline__ u64 fma2_rz_ftz(u64 a, u64 b, u64 c) {
   asm("fma.rz.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
   return d;
 }
-__device__ __forceinline__ u64 fma2_rm(u64 a, u64 b, u64 c) {
-  u64 d;
-  asm("fma.rm.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ u64 fma2_rp(u64 a, u64 b, u64 c) {
-  u64 d;
-  asm("fma.rp.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
 __device__ __forceinline__ u64 fma2_rn(u64 a, u64 b, u64 c) {
   u64 d;
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
@@ -697,43 +692,30 @@ __device__ __forceinline__ u64 fma2_rn_ftz(u64 a, u64 b, u64 c) {
   asm("fma.rn.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
   return d;
 }
-__device__ __forceinline__ u64 mul2_rn(u64 a, u64 b) {  // IEEE
-  u64 d;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-__device__ __forceinline__ u64 add2_rn(u64 a, u64 b) {
-  u64 d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-// Nearest-even cut of a pair of binary32 values to M mantissa bits on the FP32 pipe: adding
-// K = 1.5 * 2^(23-M) * 2^e (e the value's own exponent, same sign) moves the value into a binade whose unit in
-// the last place is the target grid step, so the addition itself rounds to nearest-even; K/ulp is even, so the
-// tie rule carries over; subtracting K is exact.  `v` may carry a sticky last bit (round-to-odd image of a
-// longer exact value), which keeps the result that of rounding the exact value once (needs M <= 21).
-// `kc` = {1.5 * 2^(23-M)} x 2, `neg1` = {-1} x 2.  FTZ picks whether a subnormal result is flushed.
-template <bool FTZ>
-__device__ __forceinline__ u64 rne2_fp(u64 v, u64 kc, u64 neg1) {
+// Nearest-even cut of a pair of binary32 values to M mantissa bits on the FP32 pipe.  With e the value's own
+// exponent, K = 1.5 * 2^(23-M) * 2^e (same sign) moves the value into a binade whose unit in the last place is the
+// target grid step, so the addition v + K itself rounds to nearest-even on that grid (K/ulp is even, so ties carry
+// over); subtracting K again is exact.  k0 = +-1.5 * 2^e is one logic operation per value (sign and exponent
+// kept, mantissa set to 1.5), and both steps are one packed FMA each: r = k0 * ks + v, result = k0 * (-ks) + r
+// with ks = 2^(23-M).  A zero stays zero (k0 is then a subnormal; r = k0 * ks is cancelled exactly).  Needs M <= 21
+// and exponent headroom for K, which the host checks.  `v` must be exact (or the correctly rounded binary32 image
+// of a sum whose rounding cannot decide an M-bit tie; see the host's conditions for the packed nearest-even path).
+__device__ __forceinline__ u64 rne2_fp(u64 v, u64 ks, u64 nks) {
   uint32_t lo, hi;
   asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
-  u64 e;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(e) : "r"(lo & 0xFF800000u), "r"(hi & 0xFF800000u));
-  const u64 k = mul2_rn(e, kc);
-  const u64 r = add2_rn(v, k);
-  return FTZ ? fma2_rn_ftz(k, neg1, r) : fma2_rn(k, neg1, r);
+  u64 k0;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(k0) : "r"((lo & 0xFF800000u) | 0x00400000u), "r"((hi & 0xFF800000u) | 0x00400000u));
+  const u64 r = fma2_rn(k0, ks, v);
+  return fma2_rn(k0, nks, r);
 }
-// round-to-odd image of the exact a*b+c: the toward-zero result with its last bit set when the sum is inexact
-// (the downward and upward results then differ, and they differ in the last bit).  tz carries the flush: a sum
-// below the smallest normal reads as (signed) zero, with at most the sticky bit on top.
-__device__ __forceinline__ u64 fma2_round_to_odd_ftz(u64 a, u64 b, u64 c) {
-  const u64 tz = fma2_rz_ftz(a, b, c), tm = fma2_rm(a, b, c), tp = fma2_rp(a, b, c);
-  uint32_t zl, zh, ml, mh, pl, ph;
-  asm("mov.b64 {%0, %1}, %2;" : "=r"(zl), "=r"(zh) : "l"(tz));
-  asm("mov.b64 {%0, %1}, %2;" : "=r"(ml), "=r"(mh) : "l"(tm));
-  asm("mov.b64 {%0, %1}, %2;" : "=r"(pl), "=r"(ph) : "l"(tp));
+__device__ __forceinline__ u64 mul2_rn_ftz(u64 a, u64 b) {
   u64 d;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(zl | ((ml ^ pl) & 1u)), "r"(zh | ((mh ^ ph) & 1u)));
+  asm("mul.rn.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ u64 add2_rn_ftz(u64 a, u64 b) {
+  u64 d;
+  asm("add.rn.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
 __device__ __forceinline__ u64 mul2_rz_ftz(u64 a, u64 b) {
@@ -792,7 +774,8 @@ __host__ __device__ constexpr int packed_tmem_cols() {
 enum PackedProd { PQ_NONE = 0, PQ_MASK = 1, PQ_MASK_SAT = 2 };
 
 // RNE: nearest-even instead of floor (then PQ_MASK means "round the product to M_prod bits").  Nearest-even
-// can raise a magnitude, so the slab-level proof that the clamp is idle is not used: it always clamps.
+// can raise a magnitude by half a grid step per rounding, so the slab-level proof that the clamp is idle carries a
+// growth factor for the roundings of a slab and a limit that keeps every sum at or below R_OF.
 //
 // STE = 1 (floor, sequential or chunk-16 order): instead of the sums the kernel writes the overflow masks of the
 // straight-through estimator STE^OF (App. D; layout as in the scalar tracking kernel).  The proof that lets a
@@ -883,7 +866,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
             else Bs[buf][q * 4 + j][r - BM] = s;
           }
         }
-        if (!RNE) {
+        {
           const unsigned m = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(n2 * p.nrm_scale));
           if ((tid & 31) == 0) atomicMax(&nrm[cell][is_a ? 0 : 1], m);
         }
@@ -909,8 +892,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
   const float sat = p.qa.sat;
   const uint32_t pmask = p.qp.mask;
   const float psat = p.qp.sat;
-  const u64 kc_acc = pack2(p.rne_k_acc, p.rne_k_acc), kc_prod = pack2(p.rne_k_prod, p.rne_k_prod);
-  const u64 neg1 = pack2(-1.0f, -1.0f);
+  const u64 ks_acc = pack2(p.rne_k_acc, p.rne_k_acc), nks_acc = pack2(-p.rne_k_acc, -p.rne_k_acc);
+  const u64 ks_prod = pack2(p.rne_k_prod, p.rne_k_prod), nks_prod = pack2(-p.rne_k_prod, -p.rne_k_prod);
 
   // one slab of 16 k-steps; CLAMP selects whether the magnitude clamp of Eq. 2 is applied.  The clamped
   // variant is the rare one and stays a rolled loop.  In chunk-16 order the slab starts a chunk: its first
@@ -919,7 +902,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
   auto slab_body = [&](int buf, auto clamp_tag) {
     constexpr bool CLAMP = decltype(clamp_tag)::value;
     constexpr bool REC = CLAMP && STE != 0;
-    constexpr int UNR = (CLAMP && !RNE) ? 1 : KUNROLL;
+    constexpr int UNR = CLAMP ? 1 : (RNE ? 4 : KUNROLL);  // nearest-even: a four-step body keeps the loop in the instruction cache
     if constexpr (REC) {
 #pragma unroll
       for (int i = 0; i < TM; ++i)
@@ -996,20 +979,29 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
       for (int i = 0; i < TM; ++i)
 #pragma unroll
         for (int j = 0; j < PN; ++j) {
-          // nearest-even (the floor path has left the loop body above)
+          // nearest-even (the floor path has left the loop body above).  The sum is formed by one packed FMA rounded to
+          // nearest: whenever that rounding is inexact the smaller operand lies so far below the larger one (which is
+          // on the accumulator's grid) that neither the exact sum nor its binary32 image can reach a tie of the M-bit
+          // grid, so rounding the image equals rounding the exact sum (the host admits only formats for which this holds).
+          // `.ftz` flushes exactly the sums below R_UF_acc: such a sum is a short dyadic number and survives as a subnormal.
           u64 pr = mul2_ftz(a2[i], b2[j]);
           if (PQ != PQ_NONE) {  // nearest-even on the exact product, then its saturation
-            pr = rne2_fp<false>(pr, kc_prod, neg1);
+            pr = rne2_fp(pr, ks_prod, nks_prod);
             if (PQ == PQ_MASK_SAT) {
               float plo, phi;
               unpack2(pr, plo, phi);
               pr = pack2(clamp_mag(plo, psat), clamp_mag(phi, psat));
             }
           }
-          const u64 ro = fma2_round_to_odd_ftz(pr, cc2, (CH16 && kk == 0) ? 0ull : acc1[i][j]);
+          const u64 v = (CH16 && kk == 0) ? mul2_rn_ftz(pr, cc2) : fma2_rn_ftz(pr, cc2, acc1[i][j]);
           float lo, hi;
-          unpack2(rne2_fp<true>(ro, kc_acc, neg1), lo, hi);
-          acc1[i][j] = pack2(clamp_mag(lo, sat), clamp_mag(hi, sat));
+          const u64 q = rne2_fp(v, ks_acc, nks_acc);
+          if (CLAMP) {
+            unpack2(q, lo, hi);
+            acc1[i][j] = pack2(clamp_mag(lo, sat), clamp_mag(hi, sat));
+          } else {
+            acc1[i][j] = q;
+          }
         }
       }
     }
@@ -1027,9 +1019,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
       for (int j = 0; j < PN; ++j) {
         u64& t2 = acc2[T_IN_REGS ? i : 0][T_IN_REGS ? j : 0];
         float lo, hi;
-        if (RNE) {
-          const u64 one2 = pack2(1.0f, 1.0f);
-          unpack2(rne2_fp<true>(fma2_round_to_odd_ftz(acc1[i][j], one2, t2), kc_acc, neg1), lo, hi);
+        if (RNE) {  // both operands lie on the accumulator's grid: see the note at the first hierarchy
+          unpack2(rne2_fp(add2_rn_ftz(acc1[i][j], t2), ks_acc, nks_acc), lo, hi);
         } else {
           unpack2(add2_rz_ftz(acc1[i][j], t2), lo, hi);
           lo = and_bits(lo, mask);
@@ -1239,7 +1230,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
   // a slab (or fold) whose sums provably stay below `lim` * 2^(e_max + 1) runs without the clamp: below 2^(e_max + 1)
   // the mantissa mask alone respects R_OF.  The mask variant needs more, namely that no sum reaches R_OF itself
   // (a sum in [R_OF, 2^(e_max + 1)) needs no clamp but is an overflow), so its limit is R_OF / 2^(e_max + 1)
-  const float lim = STE != 0 ? p.ste_limit : 0.999f;
+  const float lim = STE != 0 ? p.ste_limit : p.clamp_lim;
+  const float gs = p.slab_factor, gf = p.fold_factor;
   float u = 0.0f;   // upper bound of max |acc1| of this thread, as a fraction of 2^(e_max + 1)
   float u2 = 0.0f;  // chunk-16 order: the same for the second-level sums
   int slabs_in_chunk = 0;
@@ -1414,28 +1406,19 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
     if (tid < 2) nrm[cell_clear][tid] = 0u;  // read during the previous slab, filled during the next
     // ||x|| ||w|| / 2^(e_max+1), rounded up generously (the norms carry rounding errors near 2^-20)
     const float grow = sqrtf(na * nb) * 1.01f;
-    if (RNE) {
-      slab_body(buf, std::true_type());
-      if (CH16) {
-        close_chunk(std::true_type());
-      } else if (CHUNKED) {
-        if (++slabs_in_chunk == p.chunk_slabs) {
-          close_chunk(std::true_type());
-          slabs_in_chunk = 0;
-        }
-      }
-    } else if (CH16) {
+    if (CH16) {
       // the chunk starts from zero, so the CTA-wide bound alone decides (same value in every thread)
-      if (grow < lim) slab_body(buf, std::false_type());
+      const float gw = grow * gs;
+      if (gw < lim) slab_body(buf, std::false_type());
       else slab_body(buf, std::true_type());
-      if constexpr (STE != 0) ste_after_slab(s, grow < lim);
-      // |T + C| <= |T| + |C| <= u2 + grow: below 1 the mask alone already respects R_OF
+      if constexpr (STE != 0) ste_after_slab(s, gw < lim);
+      // |T + C| <= |T| + |C| <= u2 + gw: below the limit the rounding alone already respects R_OF
       const bool last = T_IN_TMEM && s + 1 == nslab;  // the final T goes to registers for the epilogue
-      if (__all_sync(0xFFFFFFFFu, u2 + grow < lim)) {
+      if (__all_sync(0xFFFFFFFFu, u2 + gw < lim)) {
         if (!T_IN_TMEM) close_chunk(std::false_type());
         else if (!last) close_chunk_tmem(std::false_type(), std::false_type());
         else close_chunk_tmem(std::false_type(), std::true_type());
-        u2 += grow;
+        u2 = (u2 + gw) * gf;
       } else {  // clamped, and the bound is refreshed from the sums
         float mx;
         if (!T_IN_TMEM) mx = close_chunk(std::true_type());
@@ -1445,8 +1428,10 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
       }
       if constexpr (STE != 0) ste_after_fold(s);
     } else {
-      bool fast = __all_sync(0xFFFFFFFFu, u + grow < lim);
-      if (!fast && u > 0.0f) {  // the carried bound may just be loose: measure |acc1|
+      bool fast = __all_sync(0xFFFFFFFFu, (u + grow) * gs < lim);
+      // the carried bound may just be loose: measure |acc1|.  The test must be the same in every lane of the warp (the
+      // vote inside is a warp-wide operation): a lane whose outputs are all zero carries u = 0 while its neighbours do not
+      if (!fast && __any_sync(0xFFFFFFFFu, u > 0.0f)) {
         float mx = 0.0f;
 #pragma unroll
         for (int i = 0; i < TM; ++i)
@@ -1457,12 +1442,12 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
             mx = fmaxf(mx, fmaxf(fabsf(lo), fabsf(hi)));
           }
         u = mx * p.inv_top;
-        fast = __all_sync(0xFFFFFFFFu, u + grow < lim);
+        fast = __all_sync(0xFFFFFFFFu, (u + grow) * gs < lim);
       }
       if (fast) slab_body(buf, std::false_type());
       else slab_body(buf, std::true_type());
       if constexpr (STE != 0) ste_after_slab(s, fast);
-      u = fminf(u + grow, 1.0f);
+      u = fminf((u + grow) * gs, 1.0f);
       if (CHUNKED) {
         if (++slabs_in_chunk == p.chunk_slabs) {
           close_chunk(std::true_type());

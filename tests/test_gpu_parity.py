@@ -122,6 +122,11 @@ def test_saturation_and_underflow_are_exercised():
         got = gpu_gemm(Apos, Bpos, one, one, None, prod, acc, order, 16).cpu().numpy()
         assert_bit_equal(got, ref_gemm(Apos, Bpos, one, one, None, prod, acc, order, 16))
         assert (got == np.float32(acc.r_of)).any()
+        for rname in ("m7e4_code_rne", "m4e4_rne"):      # nearest-even: rounds up into R_OF, never past it
+            pr, ar = FORMATS[rname]
+            got = gpu_gemm(Apos, Bpos, one, one, None, pr, ar, order, 16).cpu().numpy()
+            assert_bit_equal(got, ref_gemm(Apos, Bpos, one, one, None, pr, ar, order, 16), rname)
+            assert (got == np.float32(ar.r_of)).any() and (got <= np.float32(ar.r_of)).all()
     # mixed signs around the top: saturate, come back down, saturate negative
     Amix = Apos.clone()
     Amix[:, 512:] |= 0x80
@@ -130,11 +135,13 @@ def test_saturation_and_underflow_are_exercised():
 
 
 @pytest.mark.parametrize("tile", [0, 2, 3])
-def test_slow_climb_to_saturation_crosses_every_clamp_decision(tile):
+@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_code_rne", "m4e4_rne", "m10e6_rne"])
+def test_slow_climb_to_saturation_crosses_every_clamp_decision(tile, name):
     # small same-sign products: each chunk adds a little, so the second-level sum creeps up to R_OF over many
     # chunks.  On the way the kernel's running bound first skips the clamp, then measures the sums, then clamps
-    # for good; the sequential order does the same with its first-level bound.  All of it must stay exact.
-    prod, acc = code_domain_formats(7, 4)
+    # for good; the sequential order does the same with its first-level bound.  All of it must stay exact, for
+    # floor and for nearest-even (whose bound carries the growth of the roundings).
+    prod, acc = FORMATS[name]
     M, N, K = 96, 80, 4096
     a = (synth.gaussian((M, K), 81).abs() * 0.25 + 0.05) * torch.linspace(0.2, 1.2, M)[:, None]
     b = synth.gaussian((N, K), 82).abs() * 0.25 + 0.05
@@ -146,8 +153,8 @@ def test_slow_climb_to_saturation_crosses_every_clamp_decision(tile):
     try:
         for order, chunk in ((CHK, 16), (SEQ, 16), (CHK, 64)):
             got = gpu_gemm(A, B, one, one, None, prod, acc, order, chunk).cpu().numpy()
-            assert_bit_equal(got, ref_gemm(A, B, one, one, None, prod, acc, order, chunk), f"tile {tile} {order}/{chunk}")
-            if order == CHK and chunk == 16:
+            assert_bit_equal(got, ref_gemm(A, B, one, one, None, prod, acc, order, chunk), f"{name} tile {tile} {order}/{chunk}")
+            if order == CHK and chunk == 16 and name == "m7e4_code":
                 frac = float((got == np.float32(acc.r_of)).mean())
                 assert 0.02 < frac < 0.98, frac          # some outputs saturate, some do not
     finally:
@@ -576,8 +583,10 @@ CONV_CASES = [
 
 
 @pytest.mark.parametrize("case", CONV_CASES)
-@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_paper", "m4e4_rne"])
+@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_paper", "m4e4_rne", "m10e5", "m10e6_rne"])
 def test_conv2d_matches_direct_convolution(case, name):
+    # (the padded cases also hold slabs in which every row of a tile is zero while some outputs sit at R_OF and
+    # others, past the edge of the matrix, are zero: the clamp bookkeeping must take the same path in every lane)
     B, H, W, Cin, Cout, KH, KW, stride, pad = case
     prod, acc = FORMATS[name]
     x = synth.random_codes((B, H, W, Cin), 30)
