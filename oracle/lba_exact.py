@@ -20,6 +20,21 @@ def decode_e4m3(code: int) -> Fraction:
     return -v if s else v
 
 
+def decode_m4e3(code: int) -> Fraction:
+    """Value of a byte of the paper's W/A format (Sec. 3.1): sign, 3 exponent bits, 4 mantissa bits; Eq. 2 with
+    (M, E, b) = (4, 3, 0) gives (-1)^s 2^e (1 + m/16); the code e = m = 0 is read as zero."""
+    s, e, m = code >> 7, (code >> 4) & 7, code & 15
+    if e == 0 and m == 0:
+        return Fraction(0)
+    v = (1 + Fraction(m, 16)) * Fraction(2) ** e
+    return -v if s else v
+
+
+def decoder(prod_fmt):
+    """The byte decoder the product format names (flags bit2: M4E3 codes)."""
+    return decode_m4e3 if (prod_fmt[4] & 4) else decode_e4m3
+
+
 def r_of(M, E, b) -> Fraction:
     return Fraction(2) ** (2 ** E - b - 1) * (2 - Fraction(1, 2 ** M))
 
@@ -100,8 +115,9 @@ def fmaq(prod_fmt, acc_fmt, x: Fraction, w: Fraction, s: Fraction) -> Fraction:
 
 def dot(prod_fmt, acc_fmt, order, chunk, xcodes, wcodes) -> Fraction:
     """Eq. 8-9 (order 0) or two-hierarchy chunked accumulation (order 1) over byte codes."""
-    xs = [decode_e4m3(int(c)) for c in xcodes]
-    ws = [decode_e4m3(int(c)) for c in wcodes]
+    dec = decoder(prod_fmt)
+    xs = [dec(int(c)) for c in xcodes]
+    ws = [dec(int(c)) for c in wcodes]
     if order == 0:
         s = Fraction(0)
         for x, w in zip(xs, ws):

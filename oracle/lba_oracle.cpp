@@ -36,7 +36,12 @@
 //     chunk order, starting from 0, with Q_acc after every addition; Q_prod is
 //     not applied there; a short last chunk is allowed
 //   * inputs are OCP E4M3 bytes (4 exponent bits, bias 7, 3 mantissa bits,
-//     subnormals, max 448, codes 0x7F/0xFF are NaN and are rejected)
+//     subnormals, max 448, codes 0x7F/0xFF are NaN and are rejected), or, when the product
+//     format carries flag bit2, bytes of the paper's own W/A format "M4E3" (Sec. 3.1): sign,
+//     3 exponent bits, 4 mantissa bits, value (-1)^s 2^e (1 + m/16) as Eq. 2 gives for
+//     (M, E, b) = (4, 3, 0); Eq. 2 has no code for zero, so the code with e = m = 0 is read as
+//     zero (the magnitude 2^0 is given up); the per-tensor flex-bias 2^-b of Sec. 3.1 is the
+//     power-of-two scale the caller applies to the finished sum
 //   * convolution walks k = (kh, kw, c_in) with c_in fastest; padded taps are x = 0
 //     and still count toward the chunk position
 //   * output scaling: out = fl32(fl32(y*sa)*sb) (+ bias), outside the FMAq unit
@@ -64,7 +69,8 @@ struct lbo_fmt {
   int32_t exp_bits;  // E of Eq. 2
   int32_t bias;      // b of Eq. 2
   int32_t rounding;  // 0 = floor on magnitude, 1 = nearest, ties to even
-  int32_t flags;     // bit0: 1 = underflow flush on (Eq. 2), 0 = "excluding underflow"
+  int32_t flags;     // bit0: 1 = underflow flush on (Eq. 2), 0 = "excluding underflow";
+                     // bit2 (product format only): the input bytes are M4E3 codes, not OCP E4M3
 };
 // exp_bits = 0 selects the fixed-point quantiser of Eq. 1 instead: man_bits = B (all bits, sign included),
 // bias = b, rounding 0 = floor (toward minus infinity, the plain reading of "Floor" for a two's-complement
@@ -150,7 +156,7 @@ bool add_exact(const Dy& a, const Dy& b, Dy* out) {
   return true;
 }
 
-Dy mul_exact(const Dy& a, const Dy& b) {  // operands here are at most 4 bits each
+Dy mul_exact(const Dy& a, const Dy& b) {  // operands here are at most 5 bits each
   if (a.mag == 0 || b.mag == 0) return kZero;
   Dy r = {a.neg != b.neg, a.mag * b.mag, a.ex + b.ex};
   return normalised(r);
@@ -206,6 +212,16 @@ bool decode_e4m3(uint8_t code, Dy* out) {
   return true;
 }
 
+// The paper's W/A format (Sec. 3.1, "M4E3"): s eee mmmm, Eq. 2 with M = 4, E = 3, b = 0, i.e.
+// (-1)^s * 2^e * (1 + m/16) for e in 0..7; all 256 codes are numbers; e = m = 0 is zero.
+bool decode_m4e3(uint8_t code, Dy* out) {
+  int s = code >> 7, e = (code >> 4) & 0x7, m = code & 0xF;
+  if (e == 0 && m == 0) { *out = kZero; return true; }
+  Dy r = {s != 0, (u128)(16 + m), e - 4};   // (1 + m/16) * 2^e = (16 + m) * 2^(e-4)
+  *out = normalised(r);
+  return true;
+}
+
 // ---------------------------------------------------------------- Eq. 2
 struct Fmt {
   int M, E, b;
@@ -214,12 +230,14 @@ struct Fmt {
   Dy r_of;         // R_OF = 2^(2^E - b - 1) * (2 - 2^-M)
   bool fixed;      // Eq. 1 instead of Eq. 2: B = M bits in all, bias b
   bool wrap;       // fixed point: modulo 2^B instead of saturation
+  bool in_m4e3;    // (read from the product format) the operands are M4E3 bytes
 };
 
 int make_fmt(const lbo_fmt* f, Fmt* out) {
   if (!f) return LBO_ERR_ARG;
   out->fixed = false;
   out->wrap = false;
+  out->in_m4e3 = (f->flags & 4) != 0;
   if (f->exp_bits == 0) {  // Eq. 1
     if (f->man_bits < 2 || f->man_bits > 32 || f->rounding != 0) return LBO_ERR_FORMAT;
     if (f->bias < -64 || f->bias > 64) return LBO_ERR_FORMAT;
@@ -363,7 +381,13 @@ struct Chain {
   // one FMAq step: first <- Q_acc(Q_prod(x*w) + first)
   void fmaq_step(uint8_t xcode, uint8_t wcode) {
     Dy x, w;
-    if (!decode_e4m3(xcode, &x) || !decode_e4m3(wcode, &w)) { status = LBO_ERR_NAN_CODE; return; }
+    if (prod->in_m4e3) {
+      decode_m4e3(xcode, &x);
+      decode_m4e3(wcode, &w);
+    } else if (!decode_e4m3(xcode, &x) || !decode_e4m3(wcode, &w)) {
+      status = LBO_ERR_NAN_CODE;
+      return;
+    }
     Dy xw = mul_exact(x, w);
     Dy p = quantise(*prod, xw);
     Dy sum;
@@ -553,6 +577,14 @@ int lbo_decode_e4m3(uint8_t code, double* value) {
   if (!value) return LBO_ERR_ARG;
   Dy v;
   if (!decode_e4m3(code, &v)) return LBO_ERR_NAN_CODE;
+  return to_double(v, value) ? LBO_OK : LBO_ERR_RANGE;
+}
+
+// value of one byte of the paper's M4E3 W/A format (bias 0)
+int lbo_decode_m4e3(uint8_t code, double* value) {
+  if (!value) return LBO_ERR_ARG;
+  Dy v;
+  decode_m4e3(code, &v);
   return to_double(v, value) ? LBO_OK : LBO_ERR_RANGE;
 }
 

@@ -2,7 +2,8 @@
 
 Arrays are numpy: uint8 for E4M3 bytes, float32 for scales, bias and outputs.
 A format is a tuple ``(M, E, b, rounding, flags)`` as in Eq. 2 of the paper, with
-``rounding`` 0 = floor on the magnitude, 1 = nearest-even and ``flags`` bit0 = underflow on.
+``rounding`` 0 = floor on the magnitude, 1 = nearest-even and ``flags`` bit0 = underflow on;
+bit2 on the product format says that the input bytes are codes of the paper's M4E3 W/A format.
 """
 import ctypes as C
 import os
@@ -17,6 +18,7 @@ CHUNKED = 1
 ROUND_FLOOR = 0
 ROUND_NEAREST_EVEN = 1
 FLAG_UNDERFLOW = 1
+FLAG_INPUT_M4E3 = 4
 
 
 class OracleError(RuntimeError):
@@ -75,6 +77,12 @@ def default_threads():
 def decode_e4m3(code):
     v = C.c_double()
     _check(lib().lbo_decode_e4m3(C.c_uint8(int(code)), C.byref(v)))
+    return v.value
+
+
+def decode_m4e3(code):
+    v = C.c_double()
+    _check(lib().lbo_decode_m4e3(C.c_uint8(int(code)), C.byref(v)))
     return v.value
 
 
