@@ -52,11 +52,25 @@ typedef struct {
   int32_t bias;     /* b, -96..192                                                          */
   int32_t rounding; /* LBA_ROUND_FLOOR (the paper's, Sec. 3) or LBA_ROUND_NEAREST_EVEN      */
   int32_t flags;    /* bit0 LBA_FLAG_UNDERFLOW: 1 = flush |x| < R_UF to 0 (Eq. 2);
-                       0 = "excluding underflow" (first fine-tuning stage, Sec. 3)          */
+                       0 = "excluding underflow" (first fine-tuning stage, Sec. 3);
+                       bit2 LBA_FLAG_INPUT_M4E3, read from prod_fmt only: see below          */
 } lba_fmt;
 
 enum { LBA_ROUND_FLOOR = 0, LBA_ROUND_NEAREST_EVEN = 1 };
-enum { LBA_FLAG_UNDERFLOW = 1, LBA_FLAG_WRAP = 2 };
+enum { LBA_FLAG_UNDERFLOW = 1, LBA_FLAG_WRAP = 2, LBA_FLAG_INPUT_M4E3 = 4 };
+
+/* Input byte format.  By default both operands are OCP E4M3 bytes.  With LBA_FLAG_INPUT_M4E3 set in
+ * prod_fmt->flags (the format of the multiplier, whose inputs these are) both operands are bytes of the paper's own
+ * weight/activation format instead (Sec. 3.1: "M4E3 representation with flex-bias"): s eee mmmm, one sign bit,
+ * 3 exponent bits, 4 mantissa bits, decoded as Eq. 2 gives for (M, E, b) = (4, 3, 0):
+ *     value = (-1)^s * 2^e * (1 + m/16),  e = 0..7,  largest magnitude 248 = R_OF,
+ * except that the code with e = m = 0 (0x00, 0x80) is zero: Eq. 2 has no code for zero, and this reading gives up
+ * the magnitude 2^0 for it.  All 256 codes are numbers (no NaN).  The per-tensor flex-bias of Sec. 3.1, a power of
+ * two, is the caller's scale_a / scale_b (per tensor), applied to the finished sum like every scale.  Products of
+ * two such values carry up to 10 significant bits, so a product format with M < 9 cuts them (Q_prod of Eq. 4 acts
+ * on the mantissa, which it never does for E4M3 inputs with M >= 7).  lba_gemm, lba_gemm_batched, lba_conv2d and the
+ * host-buffer variants accept the flag with the floating-point quantisers of Eq. 2; the fixed-point formats and the
+ * straight-through-estimator entry points return LBA_ERR_FORMAT for it. */
 
 /* exp_bits = 0 selects the fixed-point quantiser Q^FIXED_{B,b} of Eq. 1 (Sec. 2.1) instead, for both formats of a
  * call or for neither (else LBA_ERR_FORMAT): man_bits = B, the number of bits including the sign, 2..24; bias = b

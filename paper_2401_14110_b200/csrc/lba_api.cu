@@ -54,11 +54,19 @@ const char* const kQmName[QM_COUNT] = {"floor_fast", "floor_full", "rne_full", "
 const char* const kOrdName[ORD_COUNT] = {"seq", "chunk_slab", "chunk_any", "chunk16"};
 const char* const kLdName[LD_COUNT] = {"gemm_vec", "conv_vec", "any"};
 
-// Largest |x*w| of two E4M3 values and the grid every product lies on.
-constexpr double kMaxProduct = 448.0 * 448.0;  // 200704
+// What the host needs to know about the operand bytes: the largest |x*w|, the grid every product (hence every sum)
+// lies on, the smallest non-zero |x*w| as a power of two at or below it, and the widest product significand.
+struct InputInfo {
+  double max_product;   // E4M3: 448^2; M4E3 (Sec. 3.1): 248^2
+  int top_product_exp;  // max_product < 2^top_product_exp
+  int grid_exp;         // every product is a multiple of 2^grid_exp
+  int min_product_exp;  // the smallest non-zero |x*w| lies in [2^min_product_exp, 2^(min_product_exp+1))
+  int product_bits;     // significant bits of a product, at most
+  int decode_exp;       // generic kernel: its byte-to-binary32 step yields value * 2^-decode_exp
+};
+constexpr InputInfo kE4M3 = {448.0 * 448.0, 18, -18, -18, 8, 120};
+constexpr InputInfo kM4E3 = {248.0 * 248.0, 16, -8, 0, 10, 0};
 constexpr double kPairEff = 0.91;              // MAC rate of the cluster-pair tile relative to the plain 64x64 tile (measured)
-constexpr int kMinProductExp = -18;            // every product, hence every sum, is a multiple of 2^-18
-constexpr int kProductBits = 8;                // significant bits of a product of two E4M3 values, at most
 
 struct Plan {
   int qm, ord;
@@ -70,6 +78,7 @@ struct Plan {
   QConst qp, qa;
   int chunk_slabs, chunk;
   int kp, ka, sx;   // product carrier = value * 2^kp, accumulator carrier = value * 2^ka, A operand = x * 2^sx
+  int in_m4e3;      // operands are M4E3 bytes
   double a_top;     // largest reachable accumulator magnitude (real domain)
   // fixed-point accumulation (Eq. 1): the integer kernel's constants
   bool fixed;
@@ -102,6 +111,8 @@ void fill_qconst(QConst* q, int M, float sat) {
 int make_fixed_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_t K, Plan* pl) {
   for (const lba_fmt* f : {pf, af})
     if (f->exp_bits != 0 || f->man_bits < 2 || f->man_bits > 24 || f->rounding != LBA_ROUND_FLOOR) return LBA_ERR_FORMAT;
+  if (pf->flags & LBA_FLAG_INPUT_M4E3) return LBA_ERR_FORMAT;  // the integer kernel decodes E4M3 only
+  const double kMaxProduct = kE4M3.max_product;
   if (order != LBA_ORDER_SEQUENTIAL && order != LBA_ORDER_CHUNKED) return LBA_ERR_ORDER;
   if (order == LBA_ORDER_CHUNKED && chunk < 1) return LBA_ERR_ORDER;
   // the product P * 2^(qx + qw), qx + qw in [-18, 10], is cut by a right shift of 22 - b_prod - qx - qw >= 0
@@ -146,15 +157,21 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
   if (order != LBA_ORDER_SEQUENTIAL && order != LBA_ORDER_CHUNKED) return LBA_ERR_ORDER;
   if (order == LBA_ORDER_CHUNKED && chunk < 1) return LBA_ERR_ORDER;
   const bool nearest = af->rounding == LBA_ROUND_NEAREST_EVEN;
+  const InputInfo in = (pf->flags & LBA_FLAG_INPUT_M4E3) ? kM4E3 : kE4M3;
+  const double kMaxProduct = in.max_product;
+  pl->in_m4e3 = (pf->flags & LBA_FLAG_INPUT_M4E3) ? 1 : 0;
 
   // ---- Q_prod
-  const bool p_flush = (pf->flags & LBA_FLAG_UNDERFLOW) && pf->bias < -kMinProductExp;  // R_UF_prod > 2^-18
-  const int kp = p_flush ? pf->bias - 126 : -108;  // carrier = value * 2^kp; 2^-18 * 2^-108 is still normal
+  // the flush is reachable iff R_UF_prod = 2^-b exceeds the smallest non-zero product
+  const bool p_flush = (pf->flags & LBA_FLAG_UNDERFLOW) && -pf->bias > in.min_product_exp;
+  // carrier = value * 2^kp; without a flush the grid step 2^grid_exp is placed at the smallest normal number
+  const int no_flush_carrier = -126 - in.grid_exp;
+  const int kp = p_flush ? pf->bias - 126 : no_flush_carrier;
   const double p_rof = r_of(pf);
   // nearest-even can carry a value in the last half step below R_OF past it, so reachability
   // is assessed with that margin; floor never increases a magnitude
   const bool p_sat = p_rof <= kMaxProduct * (nearest ? 1.0 + std::ldexp(1.0, -pf->man_bits - 1) : 1.0);
-  const bool p_round = pf->man_bits < 7;  // an E4M3 product has at most 8 significant bits
+  const bool p_round = pf->man_bits < in.product_bits - 1;  // an E4M3 product has at most 8 significant bits, an M4E3 one 10
   const int p_emax = (1 << pf->exp_bits) - pf->bias - 1;
   float p_sat_carrier = FLT_MAX;
   if (p_sat) {
@@ -162,8 +179,9 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
     p_sat_carrier = (float)std::ldexp(p_rof, kp);
   }
   // ---- Q_acc
-  const bool a_flush = (af->flags & LBA_FLAG_UNDERFLOW) && af->bias < -kMinProductExp;
-  const int ka = a_flush ? af->bias - 126 : -108;
+  // a sum can cancel down to one grid step: the flush is reachable iff R_UF_acc exceeds it
+  const bool a_flush = (af->flags & LBA_FLAG_UNDERFLOW) && -af->bias > in.grid_exp;
+  const int ka = a_flush ? af->bias - 126 : no_flush_carrier;
   const double a_rof = r_of(af);
   const double max_term = p_sat ? p_rof : kMaxProduct;
   // |S_i| <= i * max_term under floor; under nearest-even each step may add half a grid step
@@ -204,8 +222,8 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
   pl->ka = ka;
   pl->sx = sx;
   pl->a_top = a_sat ? a_rof : max_sum;
-  pl->dec_a = (float)std::ldexp(1.0, 120 + sx);
-  pl->dec_b = (float)std::ldexp(1.0, 120 + sw);
+  pl->dec_a = (float)std::ldexp(1.0, in.decode_exp + sx);
+  pl->dec_b = (float)std::ldexp(1.0, in.decode_exp + sw);
   pl->c = (float)std::ldexp(1.0, ka - kp);
   const int u1 = (-ka) / 2, u2 = (-ka) - u1;
   pl->un1 = (float)std::ldexp(1.0, u1);
@@ -261,8 +279,8 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
   pl->rne_packed = 0;
   if (pl->qm == QM_RNE_FULL) {
     const int top_acc = (a_sat ? a_emax + 1 : (int)std::ceil(std::log2(max_sum)) + 1) + ka;
-    const int top_prod = 18 + kp;
-    const int prod_bits = pf->man_bits + 1 < kProductBits ? pf->man_bits + 1 : kProductBits;
+    const int top_prod = in.top_product_exp + kp;
+    const int prod_bits = pf->man_bits + 1 < in.product_bits ? pf->man_bits + 1 : in.product_bits;
     pl->rne_packed = (top_acc + 25 - af->man_bits <= 127) && (top_prod + 25 - pf->man_bits <= 127) && af->man_bits <= 10 &&
                      prod_bits <= af->man_bits + 1 && ka - kp >= -12 && ka - kp <= 60;
   }
@@ -365,6 +383,7 @@ void apply_plan(Problem* p, const Plan& pl) {
   p->fold_factor = pl.fold_factor;
   p->pq = pl.pq;
   p->rne_packed = pl.rne_packed;
+  p->in_m4e3 = pl.in_m4e3;
   p->rne_k_acc = pl.rne_k_acc;
   p->rne_k_prod = pl.rne_k_prod;
   p->fx_shift0 = pl.fx_shift0;
@@ -535,7 +554,7 @@ int lba_gemm_last_overflow(const uint8_t* A, const uint8_t* B, int64_t M, int64_
   Plan pl;
   const int st = make_plan(prod_fmt, acc_fmt, LBA_ORDER_SEQUENTIAL, 1, K, &pl);
   if (st != LBA_OK) return st;
-  if (pl.fixed || (pl.qm != QM_FLOOR_FAST && pl.qm != QM_FLOOR_FULL)) return LBA_ERR_FORMAT;  // Eq. 2, floor rounding only
+  if (pl.fixed || pl.in_m4e3 || (pl.qm != QM_FLOOR_FAST && pl.qm != QM_FLOOR_FULL)) return LBA_ERR_FORMAT;  // Eq. 2, floor rounding, E4M3 operands
   if (M == 0 || N == 0) return LBA_OK;
   if (!last || (K > 0 && (!A || !B))) return LBA_ERR_NULL;
   if ((N + 63) / 64 > 65535) return LBA_ERR_SHAPE;
@@ -562,7 +581,7 @@ int lba_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, 
   Plan pl;
   const int st = make_plan(prod_fmt, acc_fmt, order, chunk, K, &pl);
   if (st != LBA_OK) return st;
-  if (pl.fixed || (pl.qm != QM_FLOOR_FAST && pl.qm != QM_FLOOR_FULL)) return LBA_ERR_FORMAT;  // Eq. 2, floor rounding only
+  if (pl.fixed || pl.in_m4e3 || (pl.qm != QM_FLOOR_FAST && pl.qm != QM_FLOOR_FULL)) return LBA_ERR_FORMAT;  // Eq. 2, floor rounding, E4M3 operands
   const bool chunked = order == LBA_ORDER_CHUNKED;
   const int64_t chunks = chunked ? (K + chunk - 1) / chunk : 0;
   Problem p;

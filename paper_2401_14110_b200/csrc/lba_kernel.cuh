@@ -73,7 +73,8 @@ struct Problem {
   float nrm_scale;     // 2^-(e_max_acc + 1), or 0 when the accumulator cannot saturate
   float inv_top;       // accumulator carrier -> fraction of 2^(e_max_acc + 1)
   int pq;              // PackedProd: what Q_prod does beyond the flush
-  int rne_packed;      // nearest-even: 1 if the packed kernel's exponent headroom suffices
+  int rne_packed;      // nearest-even: 1 if the packed kernel's conditions hold (see the host plan)
+  int in_m4e3;         // operands are bytes of the paper's M4E3 W/A format (Sec. 3.1) instead of OCP E4M3
   float rne_k_acc, rne_k_prod;  // 2^(23 - M) for the accumulator and the product format
   // clamp elision: a slab or fold runs without the magnitude clamp while (bound + growth) * factor < clamp_lim.
   // Floor never raises a magnitude: factors 1, limit just under 1 (of 2^(e_max+1)).  Nearest-even can raise one by
@@ -183,6 +184,15 @@ __device__ __forceinline__ float decode_e4m3_top(uint32_t top, float mul) {
   float mag = __uint_as_float((top >> 4) & 0x07F00000u);
   float v = mul_ieee(mag, mul);
   return __uint_as_float(__float_as_uint(v) | (top & 0x80000000u));
+}
+
+// Byte of the paper's W/A format (Sec. 3.1; s eee mmmm, held in the top byte of `top`) -> its value
+// (-1)^s 2^e (1 + m/16): the seven magnitude bits, moved to the low exponent and high mantissa bits of a binary32
+// pattern and added to the pattern of 1.0, are that number; the code e = m = 0 is zero.
+__device__ __forceinline__ float decode_m4e3_top(uint32_t top) {
+  const uint32_t mag = (top >> 5) & 0x03F80000u;
+  const uint32_t bits = mag ? mag + 0x3F800000u : 0u;
+  return __uint_as_float(bits | (top & 0x80000000u));
 }
 
 __device__ __forceinline__ uint32_t byte_to_top(uint32_t word, int j) {  // j in 0..3
@@ -377,7 +387,10 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), TRACK == TRACK_MASK_DIF
         const int stride = is_a ? BM : BN;
         const uint32_t w4[4] = {raw[l].x, raw[l].y, raw[l].z, raw[l].w};
 #pragma unroll
-        for (int j = 0; j < BK; ++j) dst[j * stride] = decode_e4m3_top(byte_to_top(w4[j >> 2], j & 3), mul);
+        for (int j = 0; j < BK; ++j) {
+          const uint32_t top = byte_to_top(w4[j >> 2], j & 3);
+          dst[j * stride] = p.in_m4e3 ? mul_ieee(decode_m4e3_top(top), mul) : decode_e4m3_top(top, mul);
+        }
       }
     }
   };
@@ -856,8 +869,13 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           float v[4];
-          e4m3x2_to_f32(w4[q], v[0], v[1]);
-          e4m3x2_to_f32(w4[q] >> 16, v[2], v[3]);
+          if (p.in_m4e3) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = decode_m4e3_top(byte_to_top(w4[q], j));
+          } else {
+            e4m3x2_to_f32(w4[q], v[0], v[1]);
+            e4m3x2_to_f32(w4[q] >> 16, v[2], v[3]);
+          }
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             n2 = fma_rn(v[j], v[j], n2);

@@ -5,6 +5,7 @@ ROUND_FLOOR = 0          # floor on the magnitude: the paper's choice (Sec. 3)
 ROUND_NEAREST_EVEN = 1   # a parameter of the benchmark's format sweep, not the paper's choice
 FLAG_UNDERFLOW = 1       # bit0 of flags: the |x| < R_UF -> 0 branch of Eq. 2 is active
 FLAG_WRAP = 2            # bit1 of flags, fixed-point formats: two's-complement wrap-around instead of saturation
+FLAG_INPUT_M4E3 = 4      # bit2 of the product format's flags: operands are bytes of the paper's M4E3 W/A format (Sec. 3.1)
 
 ORDER_SEQUENTIAL = 0     # Eq. 8-9
 ORDER_CHUNKED = 1        # two hierarchies, Sec. 3 / App. D
@@ -47,6 +48,23 @@ def code_domain_formats(man_bits: int = 7, exp_bits: int = 4, rounding: int = RO
         half_log += 1
         c //= 4
     prod = LbaFormat(man_bits, exp_bits, b_prod, rounding, flags)
+    acc = LbaFormat(man_bits, exp_bits, b_prod - half_log, rounding, flags)
+    return prod, acc
+
+
+def m4e3_input_formats(man_bits: int = 7, exp_bits: int = 4, rounding: int = ROUND_FLOOR,
+                       flags: int = FLAG_UNDERFLOW, chunk: int = PAPER_CHUNK):
+    """(prod_fmt, acc_fmt) for FMAq on code values of the paper's own W/A format (M4E3, largest magnitude 248).
+
+    The same two rules as ``code_domain_formats``: b_prod is the largest bias for which the largest product, 248^2,
+    stays below R_OF, i.e. 2^E - 16, and b_acc = b_prod - log2(chunk)/2.  The product format carries the input flag."""
+    b_prod = 2 ** exp_bits - 16
+    half_log = 0
+    c = chunk
+    while c >= 4:
+        half_log += 1
+        c //= 4
+    prod = LbaFormat(man_bits, exp_bits, b_prod, rounding, flags | FLAG_INPUT_M4E3)
     acc = LbaFormat(man_bits, exp_bits, b_prod - half_log, rounding, flags)
     return prod, acc
 

@@ -57,6 +57,47 @@ def e4m3_decode(codes: torch.Tensor) -> torch.Tensor:
     return codes.view(torch.float8_e4m3fn).to(torch.float32)
 
 
+M4E3_MAX = 248.0
+
+
+def m4e3_encode(t: torch.Tensor) -> torch.Tensor:
+    """float32 tensor -> uint8 codes of the paper's W/A byte format (s eee mmmm, magnitudes 2^e (1 + m/16), e = 0..7,
+    the code e = m = 0 being zero): magnitudes are clamped to 248, rounded to the nearest grid point (ties to the even
+    mantissa), and those below 1 become zero; the magnitude 1, whose code means zero, is moved up to 1.0625.
+    (The paper rounds stochastically while training; this generator only has to land on the grid.)"""
+    t = t.detach().to(torch.float32)
+    mag = t.abs().clamp(max=M4E3_MAX)
+    e = torch.floor(torch.log2(mag.clamp_min(1.0))).clamp(0, 7)
+    step = torch.exp2(e) / 16.0
+    q = torch.round(mag / step) * step                      # torch.round: ties to even
+    e2 = torch.floor(torch.log2(q.clamp_min(1.0))).clamp(0, 7)   # rounding may have carried into the next binade
+    m = torch.round(q / torch.exp2(e2) * 16.0 - 16.0).clamp(0, 15)
+    code = (e2.to(torch.int32) << 4) | m.to(torch.int32)
+    code = torch.where(code == 0, torch.ones_like(code), code)   # magnitude 1 -> 1.0625
+    code = torch.where(mag < 1.0, torch.zeros_like(code), code)
+    code = code | ((t < 0) & (code != 0)).to(torch.int32) * 0x80
+    return code.to(torch.uint8)
+
+
+def m4e3_decode(codes: torch.Tensor) -> torch.Tensor:
+    """uint8 codes of the paper's W/A byte format -> float32 values (used to build inputs and glue only)."""
+    c = codes.to(torch.int32)
+    mag = torch.exp2(((c >> 4) & 7).to(torch.float32)) * (1.0 + (c & 15).to(torch.float32) / 16.0)
+    mag = torch.where((c & 0x7F) == 0, torch.zeros_like(mag), mag)
+    return torch.where((c & 0x80) != 0, -mag, mag)
+
+
+def quantise_m4e3_per_tensor(t: torch.Tensor):
+    """(codes, scale[1]) in the paper's flex-bias W/A format (Sec. 3.1): one power-of-two scale per tensor, the
+    smallest that keeps the largest magnitude at or below 248 (the largest integer bias that prevents overflow)."""
+    absmax = float(t.detach().abs().max())
+    exp = int(np.ceil(np.log2(max(absmax, 1e-30) / M4E3_MAX)))
+    if absmax / 2.0 ** exp > M4E3_MAX:
+        exp += 1
+    scale = torch.tensor([2.0 ** exp], dtype=torch.float32, device=t.device)
+    return m4e3_encode(t / scale), scale
+
+
 def quantise_per_tensor(t: torch.Tensor):
     """(codes, scale[1]) with scale = absmax/448 so the largest magnitude maps to 448."""
     absmax = t.detach().abs().max().to(torch.float32)

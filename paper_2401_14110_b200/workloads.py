@@ -113,15 +113,27 @@ class LbaCall:
         return m * n * k * (self.x.shape[0] if self.kind == "bgemm" else 1)
 
 
-def _quant_act(t_nhwc: torch.Tensor):
+def _quant_act(t_nhwc: torch.Tensor, wa_format: str = "e4m3"):
+    if wa_format == "m4e3":
+        codes, scale = synth.quantise_m4e3_per_tensor(t_nhwc)
+        return codes.to(t_nhwc.device).contiguous(), scale.to(t_nhwc.device)
     codes, scale = synth.quantise_per_tensor(t_nhwc)
     return codes.contiguous(), scale.to(t_nhwc.device)
 
 
-def build_resnet_calls(arch: str, batch: int, config: int, device, conv_fn, gemm_fn, image_hw: int = 224):
+def _quant_weight(w: torch.Tensor, wa_format: str = "e4m3"):
+    if wa_format == "m4e3":      # the paper's flex-bias: one power-of-two scale per tensor (Sec. 3.1)
+        return synth.quantise_m4e3_per_tensor(w)
+    return synth.quantise_per_channel(w)
+
+
+def build_resnet_calls(arch: str, batch: int, config: int, device, conv_fn, gemm_fn, image_hw: int = 224,
+                       wa_format: str = "e4m3"):
     """Run one forward pass of ResNet-18/50 through ``conv_fn``/``gemm_fn`` and record every LBA call.
 
     conv_fn(x, w, sx, sw, stride, pad) -> float32 NHWC output; gemm_fn(a, b, sa, sb) -> float32 [M][N].
+    ``wa_format``: "e4m3" (OCP E4M3 bytes, per-tensor activation and per-channel weight scales) or "m4e3" (the paper's
+    own W/A bytes with one power-of-two flex-bias scale per tensor, Sec. 3.1).
     Returns the list of LbaCall (operands on ``device``) and the logits.
     """
     specs = {"resnet18": resnet18_convs, "resnet50": resnet50_convs}[arch]()
@@ -135,11 +147,11 @@ def build_resnet_calls(arch: str, batch: int, config: int, device, conv_fn, gemm
         index += 1
         w = synth.he_normal((spec.c_out, spec.k, spec.k, spec.c_in), spec.k * spec.k * spec.c_in,
                             synth.seed_for(config, 100 + index))
-        codes, scale = synth.quantise_per_channel(w)
+        codes, scale = _quant_weight(w, wa_format)
         return codes.to(device), scale.to(device)
 
     def run_conv(spec, act):
-        xc, sx = _quant_act(act)
+        xc, sx = _quant_act(act, wa_format)
         wc, sw = weights(spec)
         call = LbaCall(spec.name, "conv", xc, wc, sx, sw, (spec.stride, spec.stride), (spec.pad, spec.pad))
         calls.append(call)
@@ -168,8 +180,8 @@ def build_resnet_calls(arch: str, batch: int, config: int, device, conv_fn, gemm
     pooled = act.mean(dim=(1, 2))                                  # [B][C]
     c = pooled.shape[1]
     fc_w = synth.gaussian((1000, c), synth.seed_for(config, 99), std=float((1.0 / c) ** 0.5))
-    wc, sw = synth.quantise_per_channel(fc_w)
-    xc, sx = _quant_act(pooled)
+    wc, sw = _quant_weight(fc_w, wa_format)
+    xc, sx = _quant_act(pooled, wa_format)
     call = LbaCall("fc", "gemm", xc, wc.to(device), sx, sw.to(device))
     calls.append(call)
     logits = gemm_fn(xc, call.w, sx, call.sw)

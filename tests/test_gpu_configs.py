@@ -11,7 +11,7 @@ import torch
 from oracle import lba_oracle as orc
 from paper_2401_14110_b200 import binding as lba
 from paper_2401_14110_b200 import synth, workloads
-from paper_2401_14110_b200 import code_domain_formats, fixed_point_format, ORDER_SEQUENTIAL as SEQ, ORDER_CHUNKED as CHK
+from paper_2401_14110_b200 import code_domain_formats, m4e3_input_formats, fixed_point_format, ORDER_SEQUENTIAL as SEQ, ORDER_CHUNKED as CHK
 
 pytestmark = pytest.mark.gpu
 
@@ -70,8 +70,8 @@ def _check_call(call, prod, acc, order, tiles, seed):
     return out
 
 
-def _resnet(arch, batch, config, tiles):
-    prod, acc = code_domain_formats(7, 4)
+def _resnet(arch, batch, config, tiles, wa_format="e4m3"):
+    prod, acc = code_domain_formats(7, 4) if wa_format == "e4m3" else m4e3_input_formats(7, 4)
 
     def conv_fn(x, w, sx, sw, stride, pad):
         return lba.lba_conv2d(x, w, sx, sw, None, stride, pad, prod, acc, CHK, 16)
@@ -79,7 +79,7 @@ def _resnet(arch, batch, config, tiles):
     def gemm_fn(a, b, sa, sb):
         return lba.lba_gemm(a, b, sa, sb, None, prod, acc, CHK, 16)
 
-    calls, logits = workloads.build_resnet_calls(arch, batch, config, DEV, conv_fn, gemm_fn)
+    calls, logits = workloads.build_resnet_calls(arch, batch, config, DEV, conv_fn, gemm_fn, wa_format=wa_format)
     assert torch.isfinite(logits).all()
     for i, call in enumerate(calls):
         _check_call(call, prod, acc, CHK, tiles, 1000 * config + 10 * i)
@@ -94,6 +94,17 @@ def test_config2_resnet18_batch32_every_conv_and_fc():
     calls = _resnet("resnet18", 32, 2, tiles=64)
     assert len(calls) == 21
     assert sum(c.macs for c in calls) == 58050347008          # 1.81 GMAC per image, batch 32
+    torch.cuda.empty_cache()
+
+
+def test_resnet18_batch32_in_the_papers_own_wa_format():
+    # the forward regime of the paper's FP8 runs (Sec. 3.1, Table 3): weights and activations in the M4E3 byte format
+    # with one power-of-two flex-bias per tensor, M7E4 product and accumulator formats; products carry ten
+    # significant bits here, so Q_prod really cuts the mantissa
+    calls = _resnet("resnet18", 32, 2, tiles=32, wa_format="m4e3")
+    assert len(calls) == 21
+    prod, _ = m4e3_input_formats(7, 4)
+    assert "pq=cut" in lba.describe_plan(*calls[3].gemm_shape, prod, _, CHK, 16, is_conv=True)
     torch.cuda.empty_cache()
 
 

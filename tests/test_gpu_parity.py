@@ -6,6 +6,7 @@ import torch
 from oracle import lba_oracle as orc
 from paper_2401_14110_b200 import binding as lba
 from paper_2401_14110_b200 import synth
+from paper_2401_14110_b200 import m4e3_input_formats, FLAG_INPUT_M4E3
 from paper_2401_14110_b200 import (LbaFormat, fixed_point_format, code_domain_formats, M7E4_PAPER, WIDE, ORDER_SEQUENTIAL as SEQ,
                                    ORDER_CHUNKED as CHK)
 
@@ -539,6 +540,95 @@ def test_random_shapes_pair_tile_masks_and_fixed_point():
         order, chunk = [(SEQ, 1), (CHK, 16), (CHK, 7), (CHK, 48)][it % 4]
         assert_bit_equal(gpu_gemm(A, B, sa, sb, None, fp, fa, order, chunk), ref_gemm(A, B, sa, sb, None, fp, fa, order, chunk),
                          what + f" fixed point {fp.as_tuple()} {fa.as_tuple()} order {order} chunk {chunk}")
+
+
+M4E3_FORMATS = {
+    "m7e4": m4e3_input_formats(7, 4),                                          # the paper's FP8 runs: Q_prod cuts 10 -> 8 bits
+    "m7e4_rne": m4e3_input_formats(7, 4, rounding=1),
+    "m4e3_acc": (LbaFormat(4, 3, -8, 0, 1 | FLAG_INPUT_M4E3), LbaFormat(4, 3, -10)),   # narrow accumulator: saturates
+    "m10e5": m4e3_input_formats(10, 5),                                        # M_prod >= 9: products pass uncut
+    "m7e4_flush": (LbaFormat(7, 4, -3, 0, 1 | FLAG_INPUT_M4E3), LbaFormat(7, 4, -5)),  # R_UF_prod = 8: the product flush acts
+    "m7e4_sat": (LbaFormat(7, 4, 3, 0, 1 | FLAG_INPUT_M4E3), LbaFormat(7, 4, 1)),      # R_OF_prod = 8160: Q_prod saturates
+    "m5e4_rne_no_uf": m4e3_input_formats(5, 4, rounding=1, flags=0),
+    "m9e5_rne": m4e3_input_formats(9, 5, rounding=1),
+    "wide_rne": (LbaFormat(23, 8, 127, 1, 1 | FLAG_INPUT_M4E3), LbaFormat(23, 8, 127, 1)),
+}
+
+
+@pytest.mark.parametrize("name", list(M4E3_FORMATS))
+def test_m4e3_inputs_all_code_pairs_k1(name):
+    # the paper's own W/A byte format (Sec. 3.1): every one of the 256 x 256 code pairs through one FMAq
+    prod, acc = M4E3_FORMATS[name]
+    codes = torch.arange(256, dtype=torch.uint8)[:, None].contiguous()
+    one = torch.ones(1)
+    got = gpu_gemm(codes, codes, one, one, None, prod, acc, SEQ, 16)
+    want = ref_gemm(codes, codes, one, one, None, prod, acc, SEQ, 16)
+    assert_bit_equal(got, want, name)
+    if name == "m7e4":      # not vacuous: the mantissa cut of Q_prod changed some products
+        exact = synth.m4e3_decode(codes).double() @ synth.m4e3_decode(codes).double().T
+        assert (torch.from_numpy(want).double() != exact).any()
+
+
+@pytest.mark.parametrize("name", list(M4E3_FORMATS))
+@pytest.mark.parametrize("K", [3, 16, 47, 200, 1024])
+def test_m4e3_inputs_random_chains(name, K):
+    prod, acc = M4E3_FORMATS[name]
+    g = torch.Generator().manual_seed(900 + K)
+    A = torch.randint(0, 256, (150, K), generator=g, dtype=torch.uint8)
+    B = torch.randint(0, 256, (70, K), generator=g, dtype=torch.uint8)
+    sa = torch.tensor([2.0 ** -5])                       # the flex-bias of Sec. 3.1 is the per-tensor power-of-two scale
+    sb = torch.tensor([2.0 ** -7])
+    for order, chunk in ((SEQ, 16), (CHK, 16), (CHK, 32), (CHK, 5)):
+        got = gpu_gemm(A, B, sa, sb, None, prod, acc, order, chunk)
+        assert_bit_equal(got, ref_gemm(A, B, sa, sb, None, prod, acc, order, chunk), f"{name} K={K} {order}/{chunk}")
+
+
+@pytest.mark.parametrize("tile", [0, 1, 2, 3, 5])
+def test_m4e3_inputs_every_tile_gaussian_data(tile):
+    # Gaussian tensors quantised with a per-tensor flex-bias, ragged shapes, every CTA tile and the byte-wise loader
+    for name in ("m7e4", "m7e4_rne"):
+        prod, acc = M4E3_FORMATS[name]
+        for (M, N, K) in ((200, 100, 576), (129, 65, 147)):
+            a, sa = synth.quantise_m4e3_per_tensor(synth.gaussian((M, K), 1100 + M))
+            b, sb = synth.quantise_m4e3_per_tensor(synth.gaussian((N, K), 1200 + N, std=0.05))
+            lba.set_tile_override(tile)
+            try:
+                for order in (SEQ, CHK):
+                    got = gpu_gemm(a, b, sa, sb, None, prod, acc, order, 16)
+                    assert_bit_equal(got, ref_gemm(a, b, sa, sb, None, prod, acc, order, 16), f"{name} tile {tile} {M}x{N}x{K}")
+            finally:
+                lba.set_tile_override(-1)
+
+
+def test_m4e3_inputs_convolution_batched_and_rejections():
+    prod, acc = M4E3_FORMATS["m7e4"]
+    for case in CONV_CASES:
+        b, h, w, cin, cout, kh, kw, stride, pad = case
+        g = torch.Generator().manual_seed(77)
+        x = torch.randint(0, 256, (b, h, w, cin), generator=g, dtype=torch.uint8)
+        wt = torch.randint(0, 256, (cout, kh, kw, cin), generator=g, dtype=torch.uint8)
+        one = torch.ones(1)
+        got = lba.lba_conv2d(x.to(DEV), wt.to(DEV), one.to(DEV), one.to(DEV), None, stride, pad, prod, acc, CHK, 16)
+        want = orc.conv2d(x.numpy(), wt.numpy(), 1.0, 1.0, None, stride, pad, prod.as_tuple(), acc.as_tuple(), CHK, 16)
+        assert_bit_equal(got, want, f"m4e3 conv {case}")
+    A = torch.randint(0, 256, (3, 20, 48), dtype=torch.uint8, generator=torch.Generator().manual_seed(5)).to(DEV)
+    B = torch.randint(0, 256, (3, 30, 48), dtype=torch.uint8, generator=torch.Generator().manual_seed(6)).to(DEV)
+    one = torch.ones(1, device=DEV)
+    got = lba.lba_gemm_batched(A, B, one, one, None, prod, acc, CHK, 16)
+    for z in range(3):
+        assert_bit_equal(got[z], orc.gemm(A[z].cpu().numpy(), B[z].cpu().numpy(), 1.0, 1.0, None, prod.as_tuple(),
+                                          acc.as_tuple(), CHK, 16), f"m4e3 batched {z}")
+    # the fixed-point accumulators and the straight-through-estimator passes take E4M3 operands only
+    fx = LbaFormat(12, 0, -7, 0, FLAG_INPUT_M4E3)
+    with pytest.raises(lba.LbaError) as e:
+        lba.lba_gemm(A[0], B[0], one, one, None, fx, fixed_point_format(12, -9), SEQ, 1)
+    assert e.value.status == -3
+    with pytest.raises(lba.LbaError) as e:
+        lba.lba_gemm_ste_mask(A[0], B[0], prod, acc, CHK, 16, lba.STE_OF)
+    assert e.value.status == -3
+    with pytest.raises(lba.LbaError) as e:
+        lba.lba_gemm_last_overflow(A[0], B[0], prod, acc)
+    assert e.value.status == -3
 
 
 def test_zero_and_empty_shapes():
