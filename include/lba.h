@@ -213,7 +213,10 @@ int lba_conv2d_host(const uint8_t* x, const uint8_t* w, const float* scale_x, in
  *   - A problem with lba_gemm_host_workspace_bytes(...) > LBA_STATIC_WORKSPACE_BYTES is refused with
  *     LBA_ERR_STATIC_LIMIT and nothing is enqueued (roughly: M*K + N*K + 4*M*N must fit in 8 MiB).
  *   - The first call on each device looks up the array's device address (once, with that device
- *     current) and keeps it; make that first call outside any stream capture.
+ *     current) and keeps it; make that first call outside any stream capture.  The kept address belongs
+ *     to the device's primary context as it was then: after cudaDeviceReset (or anything else that
+ *     destroys and re-creates that context) it is stale, and this entry point must not be used again
+ *     in the same process.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left there.
  *     Nothing in it has to start at zero: each call overwrites the operand areas it reads and the
  *     kernel writes every output element before it is copied back.  Two calls whose work overlaps on

@@ -608,6 +608,31 @@ int lbo_quantise(const lbo_fmt* f, double x, double* y) {
   return to_double(quantise(fm, v), y) ? LBO_OK : LBO_ERR_RANGE;
 }
 
+// One FMAq step (Eq. 4) from given running sums: out[(t * nx + i) * nw + j] = Q_acc(Q_prod(x_i * w_j) + s_t), for
+// every running sum s_t (taken as the exact number the double holds), x code and w code.  Lets the tests take the
+// last step of a chain from every state the chain can be in.
+int lbo_fmaq_grid(const lbo_fmt* pf, const lbo_fmt* af, const uint8_t* xcodes, int64_t nx, const uint8_t* wcodes,
+                  int64_t nw, const double* s_values, int64_t ns, double* out, int nthreads) {
+  Fmt p, a;
+  int st;
+  if ((st = make_fmt(pf, &p)) != LBO_OK) return st;
+  if ((st = make_fmt(af, &a)) != LBO_OK) return st;
+  if (nx < 0 || nw < 0 || ns < 0 || (nx * nw * ns > 0 && (!xcodes || !wcodes || !s_values || !out))) return LBO_ERR_ARG;
+  return parallel_items(ns * nx, nthreads, [&](int64_t item) {
+    const int64_t t = item / nx, i = item % nx;
+    Dy s0;
+    if (!from_double(s_values[t], &s0)) return (int)LBO_ERR_ARG;
+    for (int64_t j = 0; j < nw; ++j) {
+      Chain c(&p, &a, LBO_ORDER_SEQUENTIAL, 1);
+      c.first = s0;
+      c.fmaq_step(xcodes[i], wcodes[j]);
+      if (c.status != LBO_OK) return c.status;
+      if (!to_double(c.first, &out[(t * nx + i) * nw + j])) return (int)LBO_ERR_RANGE;
+    }
+    return (int)LBO_OK;
+  });
+}
+
 // One dot product over K byte pairs (element strides in bytes).  y receives the result.
 // trace, if not null, has K entries: the first-hierarchy running sum after each step
 // (in chunked order it restarts from 0 at each chunk; the entry of a chunk's last step

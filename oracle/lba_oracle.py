@@ -116,6 +116,19 @@ def dot(prod_fmt, acc_fmt, order, chunk, x, w, trace=False):
     return (y.value, tr) if trace else y.value
 
 
+def fmaq_grid(prod_fmt, acc_fmt, xcodes, wcodes, s_values, nthreads=0):
+    """float64 [len(s_values)][len(xcodes)][len(wcodes)]: one FMAq step (Eq. 4) from every given running sum."""
+    x, xp = _u8(xcodes)
+    w, wp = _u8(wcodes)
+    sv = np.ascontiguousarray(s_values, dtype=np.float64)
+    pf, af = _fmt(prod_fmt), _fmt(acc_fmt)
+    out = np.empty((sv.size, x.size, w.size), dtype=np.float64)
+    _check(lib().lbo_fmaq_grid(C.byref(pf), C.byref(af), xp, C.c_int64(x.size), wp, C.c_int64(w.size),
+                               sv.ctypes.data_as(C.POINTER(C.c_double)), C.c_int64(sv.size),
+                               out.ctypes.data_as(C.POINTER(C.c_double)), C.c_int(nthreads or default_threads())))
+    return out
+
+
 def _scales(sa, sb, bias, la, lb):
     sa, sap = _f32(sa)
     sb, sbp = _f32(sb)

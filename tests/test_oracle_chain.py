@@ -141,19 +141,98 @@ FORMAT_PAIRS = [((7, 4, -2), (7, 4, -4)), ((7, 4, 12), (7, 4, 10)), ((4, 4, -2),
                 ((10, 6, 46), (10, 6, 44)), ((4, 3, 5), (4, 3, 5)), ((3, 4, 2), (9, 5, 9))]
 
 
+def _unit(prod, acc):
+    # counts of 2^-U with U even: operands are counts of 2^-(U/2); room for two quantisations of a cancelled sum
+    return 2 * max(9, (18 + 2 * max(prod[0], acc[0]) + 1) // 2)
+
+
+def _grid_values(fmt):
+    """Every non-negative value of Q^FLOAT_{M,E,b} (Eq. 2): 0 and 2^e (1 + n/2^M), as floats (exact for these formats)."""
+    M, E, b = fmt[:3]
+    return [0.0] + [2.0 ** e * (1 + n / 2.0 ** M) for e in range(-b, 2 ** E - b) for n in range(2 ** M)]
+
+
 @pytest.mark.parametrize("rounding", [0, 1])
-def test_brute_force_all_pairs_k1(rounding):
-    # every finite E4M3 pair through one FMAq from S = 0, against the exact-rational coding
+@pytest.mark.parametrize("flags", [1, 0])
+def test_brute_force_all_pairs_k1(rounding, flags):
+    # every finite E4M3 pair through one FMAq from S = 0, for every format pair, both roundings, with and without
+    # the underflow branch: the C++ oracle against the 64-bit integer coding (all pairs) and against the
+    # exact-rational coding (a third of the pairs)
+    from helpers import int_coding as ic
     codes = FINITE
-    for pf, af in FORMAT_PAIRS[:4]:
+    vals = [ex.decode_e4m3(int(c)) for c in codes]
+    for pf, af in FORMAT_PAIRS:
+        prod, acc = pf + (rounding, flags), af + (rounding, flags)
+        U = _unit(prod, acc)
+        got = orc.fmaq_grid(prod, acc, codes, codes, [0.0])[0]           # got[i][j] = FMAq(c_i, c_j, 0)
+        xi = np.array([ic.e4m3_int(int(c), U // 2) for c in codes], dtype=np.int64)
+        want = ic.fmaq_int(prod, acc, xi[:, None], xi[None, :], 0, U)
+        assert np.array_equal(np.ldexp(want.astype(np.float64), -U), got), (prod, acc)
+        for i in range(len(codes)):
+            for j in range(i % 3, len(codes), 3):
+                assert Fraction(float(got[i, j])) == ex.quantise(acc, ex.quantise(prod, vals[i] * vals[j])), (pf, af, i, j)
+    # the same table through the GEMM entry point (what the GPU parity test of all pairs compares with)
+    prod, acc = FORMAT_PAIRS[0][0] + (rounding, flags), FORMAT_PAIRS[0][1] + (rounding, flags)
+    out = orc.gemm(codes[:, None], codes[:, None], 1.0, 1.0, None, prod, acc, SEQ, 16)
+    assert np.array_equal(out.astype(np.float64), orc.fmaq_grid(prod, acc, codes, codes, [0.0])[0])
+
+
+@pytest.mark.parametrize("rounding", [0, 1])
+def test_last_step_of_any_short_chain_from_a_covering_set_of_running_sums(rounding):
+    # A chain of K <= 4 steps is K FMAq steps, each from a running sum S that lies on the accumulator's grid.  Instead
+    # of all 254^(2K) chains (4e9 already at K = 2), every code pair is run as one step from a covering set of S:
+    # 0, the grid values of the lowest and of the highest binade (all of them up to M = 6, 64 of each above), +-R_OF, the values just above R_UF, and every
+    # 16th grid value in between (a coarser stride for the larger grids), both signs (for the 8-bit accumulator of
+    # Sec. 4: the whole grid).  C++ oracle
+    # against the 64-bit integer coding, element by element.
+    from helpers import int_coding as ic
+    codes = FINITE
+    for pf, af in FORMAT_PAIRS:
         prod, acc = pf + (rounding, 1), af + (rounding, 1)
-        A = codes[:, None]
-        out = orc.gemm(A, A, 1.0, 1.0, None, prod, acc, SEQ, 16)     # out[i][j] = FMAq(c_i, c_j, 0)
-        vals = [ex.decode_e4m3(int(c)) for c in codes]
-        for i in range(0, len(codes)):
-            for j in range(i % 3, len(codes), 3):                    # a third of the pairs exactly checked
-                want = ex.quantise(acc, ex.quantise(prod, vals[i] * vals[j]))
-                assert Fraction(float(out[i, j])) == want, (pf, af, i, j)
+        U = _unit(prod, acc)
+        grid = _grid_values(acc)
+        per = 2 ** acc[0]
+        st = max(1, per // 64)
+        pick = set(grid[:1 + per:st]) | set(grid[-per::st]) | set(grid[1::max(16, len(grid) // 96)]) | {grid[-1], grid[1], grid[2]}
+        if len(grid) <= 600:
+            pick = set(grid)
+        s_vals = sorted(pick | {-v for v in pick})
+        # sums of products are multiples of 2^-18 at least: grid values finer than the integer unit cannot occur in a chain
+        s_vals = [v for v in s_vals if (Fraction(v) * 2 ** U).denominator == 1 and (v == 0 or abs(v) >= 2.0 ** -18)]
+        s_int = np.array([int(Fraction(v) * 2 ** U) for v in s_vals], dtype=np.int64)
+        xi = np.array([ic.e4m3_int(int(c), U // 2) for c in codes], dtype=np.int64)
+        for lo in range(0, len(s_vals), 64):
+            got = orc.fmaq_grid(prod, acc, codes, codes, s_vals[lo:lo + 64])
+            want = ic.fmaq_int(prod, acc, xi[None, :, None], xi[None, None, :], s_int[lo:lo + 64, None, None], U)
+            assert np.array_equal(np.ldexp(want.astype(np.float64), -U), got), (prod, acc, lo)
+
+
+def test_integer_coding_agrees_with_rationals_on_whole_chains_for_e4():
+    # for E = 4 every value is a count of 2^-(b+M) below 2^(16-b): a chain in plain integers, against the C++ chain
+    from helpers import int_coding as ic
+    rng = np.random.default_rng(77)
+    for (pf, af) in [FORMAT_PAIRS[0], FORMAT_PAIRS[1], FORMAT_PAIRS[2]]:
+        for rounding in (0, 1):
+            prod, acc = pf + (rounding, 1), af + (rounding, 1)
+            U = _unit(prod, acc)
+            for trial in range(30):
+                K = int(rng.integers(1, 80))
+                x = rng.choice(FINITE, K)
+                w = rng.choice(FINITE, K)
+                xs = [ic.e4m3_int(int(c), U // 2) for c in x]
+                ws = [ic.e4m3_int(int(c), U // 2) for c in w]
+                s = np.int64(0)
+                for a_, b_ in zip(xs, ws):                         # Eq. 8-9
+                    s = ic.fmaq_int(prod, acc, a_, b_, s, U)
+                assert abs(int(s)) < 2 ** 62
+                assert float(np.ldexp(float(s), -U)) == orc.dot(prod, acc, SEQ, 1, x, w)
+                t = np.int64(0)                                    # two hierarchies, chunk 16
+                for j in range(0, K, 16):
+                    c = np.int64(0)
+                    for a_, b_ in zip(xs[j:j + 16], ws[j:j + 16]):
+                        c = ic.fmaq_int(prod, acc, a_, b_, c, U)
+                    t = ic.quantise_int(c + t, *acc, U)
+                assert float(np.ldexp(float(t), -U)) == orc.dot(prod, acc, CHK, 16, x, w)
 
 
 @pytest.mark.parametrize("rounding", [0, 1])
