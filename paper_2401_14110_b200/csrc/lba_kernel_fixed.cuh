@@ -10,7 +10,9 @@
 // The host checks that none of the left shifts can leave 32 bits.
 //
 // Layout: 64 x 64 outputs per CTA, 4 x 4 per thread, 256 threads, K in slabs of 16, operands decoded once per
-// CTA into shared memory as {mantissa, shift contribution} pairs; orders and loaders as in the scalar kernel.
+// CTA into shared memory, mantissas and shift contributions in arrays of their own (a thread's four neighbouring
+// values are then one 16-byte load from consecutive addresses: as {mantissa, shift} pairs the 32-byte stride between
+// lanes put two lanes of every quarter-warp on the same banks); orders and loaders as in the scalar kernel.
 #pragma once
 #include "lba_kernel.cuh"
 
@@ -40,9 +42,11 @@ __global__ void __launch_bounds__(256) lba_fixed_kernel(const Problem p) {
   constexpr bool CHUNKED = ORD != ORD_SEQ;
   static_assert(ORD == ORD_SEQ || ORD == ORD_CHUNK_SLAB || ORD == ORD_CHUNK_ANY, "order");
 
-  // .x: mantissa (A: shifted left by 22), .y: contribution to the right-shift count
-  __shared__ __align__(16) int2 As[2][BK][BM];
-  __shared__ __align__(16) int2 Bs[2][BK][BN];
+  // m: mantissa (A: shifted left by 22), q: contribution to the right-shift count
+  __shared__ __align__(16) int Am[2][BK][BM];
+  __shared__ __align__(16) int Aq[2][BK][BM];
+  __shared__ __align__(16) int Bm[2][BK][BN];
+  __shared__ __align__(16) int Bq[2][BK][BN];
 
   const int tid = threadIdx.x;
   const int tx = tid % TX, ty = tid / TX;
@@ -60,7 +64,8 @@ __global__ void __launch_bounds__(256) lba_fixed_kernel(const Problem p) {
       const int r = tid + l * NT;
       if (r < ROWS) {
         const bool is_a = r < BM;
-        int2* dst = is_a ? &As[buf][0][r] : &Bs[buf][0][r - BM];
+        int* dm = is_a ? &Am[buf][0][r] : &Bm[buf][0][r - BM];
+        int* dq = is_a ? &Aq[buf][0][r] : &Bq[buf][0][r - BM];
         const int stride = is_a ? BM : BN;
         const uint32_t w4[4] = {raw[l].x, raw[l].y, raw[l].z, raw[l].w};
 #pragma unroll
@@ -71,7 +76,8 @@ __global__ void __launch_bounds__(256) lba_fixed_kernel(const Problem p) {
           const int q = e ? e - 10 : -9;
           if (c & 0x80u) s = -s;
           // right-shift count of the product = (22 - b_prod - qx) + (-qw)
-          dst[j * stride] = is_a ? make_int2(s << 22, p.fx_shift0 - q) : make_int2(s, -q);
+          dm[j * stride] = is_a ? s << 22 : s;
+          dq[j * stride] = is_a ? p.fx_shift0 - q : -q;
         }
       }
     }
@@ -107,16 +113,16 @@ __global__ void __launch_bounds__(256) lba_fixed_kernel(const Problem p) {
     constexpr bool UP = decltype(up_tag)::value;
     int2 a[TM], b[TN];
     {
-      const int4* src = reinterpret_cast<const int4*>(&As[buf][kk][ty * 4]);
-      const int4 v0 = src[0], v1 = src[1];
-      a[0] = make_int2(v0.x, v0.y); a[1] = make_int2(v0.z, v0.w);
-      a[2] = make_int2(v1.x, v1.y); a[3] = make_int2(v1.z, v1.w);
+      const int4 vm = *reinterpret_cast<const int4*>(&Am[buf][kk][ty * 4]);
+      const int4 vq = *reinterpret_cast<const int4*>(&Aq[buf][kk][ty * 4]);
+      a[0] = make_int2(vm.x, vq.x); a[1] = make_int2(vm.y, vq.y);
+      a[2] = make_int2(vm.z, vq.z); a[3] = make_int2(vm.w, vq.w);
     }
     {
-      const int4* src = reinterpret_cast<const int4*>(&Bs[buf][kk][tx * 4]);
-      const int4 v0 = src[0], v1 = src[1];
-      b[0] = make_int2(v0.x, v0.y); b[1] = make_int2(v0.z, v0.w);
-      b[2] = make_int2(v1.x, v1.y); b[3] = make_int2(v1.z, v1.w);
+      const int4 vm = *reinterpret_cast<const int4*>(&Bm[buf][kk][tx * 4]);
+      const int4 vq = *reinterpret_cast<const int4*>(&Bq[buf][kk][tx * 4]);
+      b[0] = make_int2(vm.x, vq.x); b[1] = make_int2(vm.y, vq.y);
+      b[2] = make_int2(vm.z, vq.z); b[3] = make_int2(vm.w, vq.w);
     }
 #pragma unroll
     for (int i = 0; i < TM; ++i)

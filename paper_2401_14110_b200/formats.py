@@ -24,14 +24,6 @@ class LbaFormat:
     def as_tuple(self):
         return (self.man_bits, self.exp_bits, self.bias, self.rounding, self.flags)
 
-    @property
-    def r_uf(self) -> float:
-        return 2.0 ** (-self.bias)
-
-    @property
-    def r_of(self) -> float:
-        return 2.0 ** (2 ** self.exp_bits - self.bias - 1) * (2.0 - 2.0 ** (-self.man_bits))
-
 
 def code_domain_formats(man_bits: int = 7, exp_bits: int = 4, rounding: int = ROUND_FLOOR,
                         flags: int = FLAG_UNDERFLOW, chunk: int = PAPER_CHUNK):

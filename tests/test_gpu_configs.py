@@ -10,6 +10,7 @@ import torch
 
 from oracle import lba_oracle as orc
 from paper_2401_14110_b200 import binding as lba
+from helpers.fmt_range import r_of, r_uf
 from paper_2401_14110_b200 import synth, workloads
 from paper_2401_14110_b200 import code_domain_formats, m4e3_input_formats, fixed_point_format, ORDER_SEQUENTIAL as SEQ, ORDER_CHUNKED as CHK
 
@@ -126,7 +127,7 @@ def test_config4_bert_base_linears_with_outlier_channels():
     a = synth.e4m3_decode(calls[0].x[:64].cpu()).numpy().astype(np.float64)
     b = synth.e4m3_decode(calls[0].w[:64].cpu()).numpy().astype(np.float64)
     p = np.abs(a[:, None, :] * b[None, :, :])
-    assert ((p > 0) & (p < prod.r_uf)).mean() > 0.01
+    assert ((p > 0) & (p < r_uf(prod))).mean() > 0.01
 
 
 SWEEP = [(m, e, r) for e in (4, 5, 6) for m in range(4, 11) for r in (0, 1)]
