@@ -51,13 +51,14 @@ MIX = {
     "rne": (4.0, 2.0, 2.0, 0.0, "0.5 FMUL2 + 0.5 FFMA2 + 1 LOP3 + 1 FFMA2 (rounding on the FP32 pipe) + 1 FMNMX"),
     "rne_cut": (6.0, 3.0, 3.0, 0.0, "as rne, plus 1 LOP3 + 1 FFMA2 for the product's rounding"),
     "rne_cut_sat": (7.0, 4.0, 3.0, 0.0, "as rne_cut, plus 1 FMNMX for the product's saturation"),
+    "rne_fused": (3.5, 2.0, 1.5, 0.0, "0.5 FFMA2 (product and sum) + 1 LOP3 + 1 FFMA2 (rounding) + 1 FMNMX"),
     "rne_wide": (1.0, 0.0, 0.0, 1.0, "1 FFMA (24-bit accumulator: one IEEE FMA per MAC)"),
     "generic": (6.0, 4.0, 0.0, 2.0, "scalar FMUL + FFMA + mask + clamp (+ product steps): the generic kernel"),
     "fixed": (6.0, 4.0, 0.0, 2.0, "2 SHF + 2 add-min/max on the logic pipe; IMAD + IADD beside them"),
     "ste_diff": (11.0, 5.0, 0.0, 6.0, "FMUL + FFMA + LOP3 + FMNMX + 3 FMUL + 2 FADD + FSETP + bit insert, scalar"),
 }
 FOLD = {  # per output per chunk: (issue, logic, packed_fp, scalar_fp)
-    "floor": (2.5, 2.0, 0.5, 0.0), "rne": (3.0, 2.0, 1.0, 0.0), "rne_wide": (1.0, 0.0, 0.0, 1.0), "generic": (4.0, 2.0, 0.0, 1.0),
+    "floor": (2.5, 2.0, 0.5, 0.0), "rne": (3.5, 2.0, 1.5, 0.0), "rne_wide": (1.0, 0.0, 0.0, 1.0), "generic": (4.0, 2.0, 0.0, 1.0),
     "fixed": (4.0, 4.0, 0.0, 0.0),
 }
 

@@ -234,7 +234,8 @@ int lba_count_nan_codes(const uint8_t* codes, int64_t n, unsigned long long* cou
 
 /* Which kernel variant a call with these arguments would run, as text, e.g.
  * "tile=64x64x16 micro=4x8 q=floor_fast pq=none kernel=packed order=chunk16 load=gemm_vec grid=128x128"
- * (pq: what Q_prod does beyond its flush -- none, cut = mantissa cut, cut_sat = cut and saturation; kernel: the
+ * (pq: what Q_prod does beyond its flush -- none, cut = mantissa cut, cut_sat = cut and saturation, fused = Q_prod is
+ * the identity on every reachable product, so product and sum are one instruction; kernel: the
  * packed two-outputs-per-instruction kernel or the generic scalar one).
  * is_conv selects the loader family; for a convolution pass M = B*H_out*W_out, N = C_out,
  * K = KH*KW*C_in and vec_ok = (C_in % 16 == 0 and pointers aligned).  Returns LBA_OK or the

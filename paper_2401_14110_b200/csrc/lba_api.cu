@@ -79,6 +79,8 @@ struct Plan {
   int chunk_slabs, chunk;
   int kp, ka, sx;   // product carrier = value * 2^kp, accumulator carrier = value * 2^ka, A operand = x * 2^sx
   int in_m4e3;      // operands are M4E3 bytes
+  int fused;        // Q_prod is the identity on every reachable product: PQ_FUSED applies (plain packed tiles)
+  float pk_b_fused; // B operand scaling for it: 2^(sw + ka - kp), so that x' w' lands in the accumulator carrier
   double a_top;     // largest reachable accumulator magnitude (real domain)
   // fixed-point accumulation (Eq. 1): the integer kernel's constants
   bool fixed;
@@ -285,6 +287,15 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
                      prod_bits <= af->man_bits + 1 && ka - kp >= -12 && ka - kp <= 60;
   }
 
+  // ---- fused product and sum: Q_prod must be the identity on every reachable product (no cut, no saturation, no
+  // product under R_UF_prod), and the rescaled B operand must stay a normal binary32 number
+  {
+    const int swf = sw + (ka - kp);
+    const bool packed_q = pl->qm == QM_FLOOR_FAST || (pl->qm == QM_RNE_FULL && pl->rne_packed);
+    pl->fused = packed_q && !p_flush && !p_sat && !p_round && swf - 9 >= -126 && swf + 9 <= 126;
+    pl->pk_b_fused = pl->fused ? (float)std::ldexp(1.0, swf) : 0.0f;
+  }
+
   // ---- order mode
   pl->chunk = chunk;
   pl->chunk_slabs = 0;
@@ -413,6 +424,13 @@ int run(const Problem& p, const Plan& pl, int load, cudaStream_t stream) {
   }
   const TileInfo ti = tile_info(tile);
   if ((p.N + ti.bn - 1) / ti.bn > 65535 || (p.M + ti.bm - 1) / ti.bm > 2147483647LL) return LBA_ERR_SHAPE;
+  if (pl.fused && pl.ord != ORD_CHUNK_ANY) {  // the plain packed tiles have the fused variant
+    Problem q = p;
+    q.pq = PQ_FUSED;
+    q.pk_b = pl.pk_b_fused;
+    const cudaError_t e = kLaunch[pl.qm][pl.ord](tile, load, q, stream);
+    return e == cudaSuccess ? LBA_OK : cuda_fail(e);
+  }
   const cudaError_t e = kLaunch[pl.qm][pl.ord](tile, load, p, stream);
   return e == cudaSuccess ? LBA_OK : cuda_fail(e);
 }
@@ -803,8 +821,9 @@ int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, 
   const bool packed = pl.ord != ORD_CHUNK_ANY &&
                       (pl.qm == QM_FLOOR_FAST || pl.qm == QM_FLOOR_FULL || (pl.qm == QM_RNE_FULL && pl.rne_packed));
   const char* const kern = packed ? "packed" : "generic";
-  const char* const pq = pl.qm == QM_FLOOR_FAST || pl.qm == QM_RNE_WIDE ? "none"
-                         : (pl.pq == PQ_MASK_SAT ? "cut_sat" : (pl.pq == PQ_MASK ? "cut" : "none"));
+  const char* const pq = (pl.fused && packed && tile != TILE_PAIR) ? "fused"
+                         : (pl.qm == QM_FLOOR_FAST || pl.qm == QM_RNE_WIDE ? "none"
+                            : (pl.pq == PQ_MASK_SAT ? "cut_sat" : (pl.pq == PQ_MASK ? "cut" : "none")));
   if (tile == TILE_PAIR) {
     if (buf && buf_len)
       std::snprintf(buf, buf_len, "tile=64x64x%d pair micro=4x8 q=%s pq=%s kernel=%s order=%s load=%s grid=%lldx%lld", BK,

@@ -784,7 +784,10 @@ __host__ __device__ constexpr int packed_tmem_cols() {
 // cost fifty registers and half the resident CTAs
 // PQ: what Q_prod has to do beyond the flush (the host proves which cases are reachable): nothing, cut the
 // mantissa (M_prod < 7), or cut and saturate (448^2 >= R_OF_prod)
-enum PackedProd { PQ_NONE = 0, PQ_MASK = 1, PQ_MASK_SAT = 2 };
+// PQ_FUSED: Q_prod is the identity on every reachable product (no cut, no saturation, and no product can fall under
+// R_UF_prod), so FMAq(x, w, S) = Q_acc(x w + S) and the product needs no instruction of its own: one packed FMA forms the
+// exact product and the sum; the B operand then carries the accumulator's scaling.
+enum PackedProd { PQ_NONE = 0, PQ_MASK = 1, PQ_MASK_SAT = 2, PQ_FUSED = 3 };
 
 // RNE: nearest-even instead of floor (then PQ_MASK means "round the product to M_prod bits").  Nearest-even
 // can raise a magnitude by half a grid step per rounding, so the slab-level proof that the clamp is idle carries a
@@ -946,7 +949,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
         // multiplies (FP32 pipe) and masks (logic pipe) of independent outputs sit side by side in the stream
         auto product = [&](u64 av, u64 bv) -> u64 {
           u64 pr = mul2_ftz(av, bv);
-          if (PQ != PQ_NONE) {  // floor of Eq. 2 on the exact product, then its saturation
+          if (PQ == PQ_MASK || PQ == PQ_MASK_SAT) {  // floor of Eq. 2 on the exact product, then its saturation
             float plo, phi;
             unpack2(pr, plo, phi);
             plo = and_bits(plo, pmask);
@@ -959,6 +962,28 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
           }
           return pr;
         };
+        if constexpr (PQ == PQ_FUSED) {
+#pragma unroll
+          for (int i = 0; i < TM; ++i)
+#pragma unroll
+            for (int j = 0; j < PN; ++j) {
+              const u64 t = (CH16 && kk == 0) ? mul2_rz_ftz(a2[i], b2[j]) : fma2_rz_ftz(a2[i], b2[j], acc1[i][j]);
+              float lo, hi;
+              unpack2(t, lo, hi);
+              lo = and_bits(lo, mask);
+              hi = and_bits(hi, mask);
+              if constexpr (REC) {
+                if (fabsf(lo) < sat) hb[i][j] |= 1u << kk;
+                if (fabsf(hi) < sat) hb[i][j] |= 0x10000u << kk;
+              }
+              if (CLAMP) {
+                lo = clamp_mag(lo, sat);
+                hi = clamp_mag(hi, sat);
+              }
+              acc1[i][j] = pack2(lo, hi);
+            }
+          continue;
+        }
         u64 pr[PN], nx[PN];
 #pragma unroll
         for (int j = 0; j < PN; ++j) pr[j] = product(a2[0], b2[j]);
@@ -1002,16 +1027,21 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
           // on the accumulator's grid) that neither the exact sum nor its binary32 image can reach a tie of the M-bit
           // grid, so rounding the image equals rounding the exact sum (the host admits only formats for which this holds).
           // `.ftz` flushes exactly the sums below R_UF_acc: such a sum is a short dyadic number and survives as a subnormal.
-          u64 pr = mul2_ftz(a2[i], b2[j]);
-          if (PQ != PQ_NONE) {  // nearest-even on the exact product, then its saturation
-            pr = rne2_fp(pr, ks_prod, nks_prod);
-            if (PQ == PQ_MASK_SAT) {
-              float plo, phi;
-              unpack2(pr, plo, phi);
-              pr = pack2(clamp_mag(plo, psat), clamp_mag(phi, psat));
+          u64 v;
+          if constexpr (PQ == PQ_FUSED) {  // Q_prod is the identity: product and sum in one FMA
+            v = (CH16 && kk == 0) ? mul2_rn_ftz(a2[i], b2[j]) : fma2_rn_ftz(a2[i], b2[j], acc1[i][j]);
+          } else {
+            u64 pr = mul2_ftz(a2[i], b2[j]);
+            if (PQ == PQ_MASK || PQ == PQ_MASK_SAT) {  // nearest-even on the exact product, then its saturation
+              pr = rne2_fp(pr, ks_prod, nks_prod);
+              if (PQ == PQ_MASK_SAT) {
+                float plo, phi;
+                unpack2(pr, plo, phi);
+                pr = pack2(clamp_mag(plo, psat), clamp_mag(phi, psat));
+              }
             }
+            v = (CH16 && kk == 0) ? mul2_rn_ftz(pr, cc2) : fma2_rn_ftz(pr, cc2, acc1[i][j]);
           }
-          const u64 v = (CH16 && kk == 0) ? mul2_rn_ftz(pr, cc2) : fma2_rn_ftz(pr, cc2, acc1[i][j]);
           float lo, hi;
           const u64 q = rne2_fp(v, ks_acc, nks_acc);
           if (CLAMP) {

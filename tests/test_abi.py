@@ -41,6 +41,10 @@ def test_plan_selection_by_format_and_order():
     assert "q=floor_full" in lba.describe_plan(64, 64, 576, *code_domain_formats(4, 4), CHK, 16)
     assert "q=rne_full" in lba.describe_plan(64, 64, 576, *code_domain_formats(7, 4, rounding=1), CHK, 16)
     assert "q=rne_wide" in lba.describe_plan(64, 64, 576, LbaFormat(23, 8, 127, 1), LbaFormat(23, 8, 127, 1), SEQ, 16)
+    assert "pq=none" in lba.describe_plan(64, 64, 576, p, a, CHK, 16)                # the product flush is reachable
+    assert "pq=fused" in lba.describe_plan(64, 64, 576, *code_domain_formats(8, 6), CHK, 16)
+    assert "pq=fused" in lba.describe_plan(64, 64, 576, *code_domain_formats(7, 4, flags=0), SEQ, 16)
+    assert "pq=cut" in lba.describe_plan(64, 64, 576, *code_domain_formats(5, 6), CHK, 16)
     assert "load=conv_vec" in lba.describe_plan(64, 64, 576, p, a, CHK, 16, is_conv=True)
     assert "load=any" in lba.describe_plan(64, 64, 147, p, a, CHK, 16, is_conv=True, vec_ok=False)
 

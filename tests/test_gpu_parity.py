@@ -44,6 +44,7 @@ FORMATS = {
     "m4e4": code_domain_formats(4, 4),                                        # Q_prod rounds
     "m10e5": code_domain_formats(10, 5),
     "m5e6": code_domain_formats(5, 6),
+    "m8e6": code_domain_formats(8, 6),                                        # no product can be cut or flushed: fused product and sum
     "m4e3_mnist": (LbaFormat(4, 3, 5), LbaFormat(4, 3, 5)),                   # Sec. 4 accumulator
     "mixed": (LbaFormat(3, 4, 2), LbaFormat(9, 5, 9)),
     "m7e4_code_rne": code_domain_formats(7, 4, rounding=1),
@@ -91,7 +92,7 @@ def test_random_codes_short_chains(name, K):
 
 
 @pytest.mark.parametrize("tile", [0, 1, 2, 3])
-@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_paper", "m4e4_rne", "wide_rne"])
+@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_paper", "m4e4_rne", "wide_rne", "m7e4_no_uf", "m10e6_rne", "m8e6"])
 def test_every_tile_shape_with_ragged_edges(tile, name):
     prod, acc = FORMATS[name]
     lba.set_tile_override(tile)
@@ -137,7 +138,7 @@ def test_saturation_and_underflow_are_exercised():
 
 
 @pytest.mark.parametrize("tile", [0, 2, 3])
-@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_code_rne", "m4e4_rne", "m10e6_rne"])
+@pytest.mark.parametrize("name", ["m7e4_code", "m7e4_code_rne", "m4e4_rne", "m10e6_rne", "m7e4_no_uf", "m8e6"])
 def test_slow_climb_to_saturation_crosses_every_clamp_decision(tile, name):
     # small same-sign products: each chunk adds a little, so the second-level sum creeps up to R_OF over many
     # chunks.  On the way the kernel's running bound first skips the clamp, then measures the sums, then clamps
