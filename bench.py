@@ -153,6 +153,10 @@ def parse_args(argv=None):
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-streams", type=int, default=12,
                     help="network workloads: streams (each with its own device workspace) the end-to-end calls are spread over")
+    ap.add_argument("--e2e-row-blocks", type=int, default=8,
+                    help="single-GEMM workloads: the end-to-end step is issued as this many row blocks (rows of the output are "
+                         "independent chains), one lba_gemm_host call each, over three streams, so that one block's copies "
+                         "overlap another block's kernel; 1 = one call")
     ap.add_argument("--force-dist", action="store_true",
                     help="initialise torch.distributed (NCCL) even for a single rank: exercises the multi-GPU plumbing "
                          "(barrier, max over ranks) on one GPU")
@@ -559,9 +563,21 @@ def end_to_end(wl, args, device, world, dist, barrier):
         h2d += hx.numel() + hw_.numel() + 4 * (hsx.numel() + hsw.numel())
         d2h += 4 * hout.numel()
         host.append((c, hx, hw_, hsx, hsw, hout))
+    whole = [(c, hout) for c, _, _, _, _, hout in host]
     # independent calls of a step are spread round-robin over a few streams, each with its own workspace: one call's
-    # copies overlap another call's kernel; a single-call step uses one stream
-    n_streams = max(1, min(args.e2e_streams, len(wl.calls)))
+    # copies overlap another call's kernel.  A single GEMM is issued as row blocks for the same reason: the rows of the
+    # output are independent chains, so each block is a complete lba_gemm_host call on its own rows (B travels with
+    # every block, which the byte counts include)
+    blocks = 1
+    if len(host) == 1 and host[0][0].kind == "gemm" and host[0][3].numel() == 1 and args.e2e_row_blocks > 1:
+        c, hx, hw_, hsx, hsw, hout = host[0]
+        m, n, k = c.gemm_shape
+        blocks = min(args.e2e_row_blocks, m)
+        spans = [sharding.shard_rows(m, blocks, r) for r in range(blocks)]
+        host = [(c, hx[a:b], hw_, hsx, hsw, hout[a:b]) for a, b in spans]
+        ws_bytes = max(lba.gemm_host_workspace_bytes(b - a, n, k, 1, hsw.numel(), False) for a, b in spans)
+        h2d = hx.numel() + blocks * (hw_.numel() + 4 * hsw.numel() + 4)
+    n_streams = max(1, min(args.e2e_streams, len(host), 3 if blocks > 1 else len(host)))
     streams = [torch.cuda.Stream(device=device) for _ in range(n_streams)]
     wss = [torch.empty(ws_bytes, dtype=torch.uint8, device=device) for _ in range(n_streams)]
     torch.cuda.synchronize()
@@ -582,10 +598,14 @@ def end_to_end(wl, args, device, world, dist, barrier):
         step()
     barrier()
     ms = sharding.max_over_ranks((time.perf_counter() - t0) * 1e3 / steps, dist, device)
+    # the host results are the device-resident step's results, bit for bit
+    wl.run_step()
+    torch.cuda.synchronize()
+    same = all(torch.equal(hout, (c.out if c.kind == "gemm" else c.out_nhwc).cpu()) for c, hout in whole)
     return {"value": sharding.whole_job_rate(wl.macs, world, ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
-            "d2h_bytes_per_step": d2h, "ms_per_step": ms, "steps": steps,
-            "api": "lba_gemm_host / lba_conv2d_host (pinned host buffers, caller-owned device workspace, "
-                   f"{n_streams} stream(s))"}
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms, "steps": steps, "equals_device_step": same,
+            "api": "lba_gemm_host / lba_conv2d_host (pinned host buffers, caller-owned device workspaces, "
+                   f"{len(host)} call(s) over {n_streams} stream(s)" + (f": {blocks} row blocks of one GEMM" if blocks > 1 else "") + ")"}
 
 
 def main(argv=None):
