@@ -181,9 +181,6 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
     p_sat_carrier = (float)std::ldexp(p_rof, kp);
   }
   // ---- Q_acc
-  // a sum can cancel down to one grid step: the flush is reachable iff R_UF_acc exceeds it
-  const bool a_flush = (af->flags & LBA_FLAG_UNDERFLOW) && -af->bias > in.grid_exp;
-  const int ka = a_flush ? af->bias - 126 : no_flush_carrier;
   const double a_rof = r_of(af);
   const double max_term = p_sat ? p_rof : kMaxProduct;
   // |S_i| <= i * max_term under floor; under nearest-even each step may add half a grid step
@@ -191,6 +188,15 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
   const double max_sum = (double)(K > 0 ? K : 1) * max_term * growth;
   const bool a_sat = a_rof <= max_sum;
   const int a_emax = (1 << af->exp_bits) - af->bias - 1;
+  // every sum is a multiple of the grid step of the products, unless a saturation put R_OF into the chain: R_OF is a
+  // multiple of 2^(e_max - M) only, of the product format where Q_prod saturates and of the accumulator's where Q_acc does
+  int sum_grid = in.grid_exp;
+  if (p_sat && p_emax - pf->man_bits < sum_grid) sum_grid = p_emax - pf->man_bits;
+  if (a_sat && a_emax - af->man_bits < sum_grid) sum_grid = a_emax - af->man_bits;
+  // a sum can cancel down to one grid step: the flush is reachable iff R_UF_acc exceeds it; without a flush the
+  // carrier places that step at the smallest normal number
+  const bool a_flush = (af->flags & LBA_FLAG_UNDERFLOW) && -af->bias > sum_grid;
+  const int ka = a_flush ? af->bias - 126 : -126 - sum_grid;
   float a_sat_carrier = FLT_MAX;
   if (a_sat) {
     if (a_emax + ka < -126 || a_emax + ka > 127) return LBA_ERR_FORMAT;
@@ -282,7 +288,9 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
   if (pl->qm == QM_RNE_FULL) {
     const int top_acc = (a_sat ? a_emax + 1 : (int)std::ceil(std::log2(max_sum)) + 1) + ka;
     const int top_prod = in.top_product_exp + kp;
-    const int prod_bits = pf->man_bits + 1 < in.product_bits ? pf->man_bits + 1 : in.product_bits;
+    // significant bits of a quantised product: the exact product's, cut to M_prod + 1; a saturated product is R_OF_prod,
+    // which has all M_prod + 1
+    const int prod_bits = (p_sat || pf->man_bits + 1 < in.product_bits) ? pf->man_bits + 1 : in.product_bits;
     pl->rne_packed = (top_acc + 25 - af->man_bits <= 127) && (top_prod + 25 - pf->man_bits <= 127) && af->man_bits <= 10 &&
                      prod_bits <= af->man_bits + 1 && ka - kp >= -12 && ka - kp <= 60;
   }

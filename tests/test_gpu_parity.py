@@ -137,6 +137,41 @@ def test_saturation_and_underflow_are_exercised():
     assert_bit_equal(got, ref_gemm(Amix, Bpos, one, one, None, prod, acc, CHK, 16))
 
 
+SEARCH_FOUND = [
+    # R_OF_acc = 16 - 2^-14 lies off the grid of the products (multiples of 2^-8): a sum that sits at R_OF and meets
+    # the product -16 leaves -2^-14, which must not be lost below the carrier's smallest normal number
+    (LbaFormat(5, 7, 21, 1, 1 | FLAG_INPUT_M4E3), LbaFormat(17, 5, 28, 1, 1)),
+    (LbaFormat(5, 7, 21, 0, 1 | FLAG_INPUT_M4E3), LbaFormat(17, 5, 28, 0, 1)),
+    (LbaFormat(12, 6, 30, 0, 1), LbaFormat(21, 5, 31, 0, 1)),
+    # Q_prod saturates to R_OF_prod, which has M_prod + 1 significant bits, more than the accumulator keeps: the sum is
+    # not one rounding of one binary32 FMA
+    (LbaFormat(20, 2, -9, 1, FLAG_INPUT_M4E3), LbaFormat(9, 8, 3, 1, 0)),
+    (LbaFormat(19, 3, 8, 1, 1), LbaFormat(8, 6, 34, 1, 1)),
+]
+
+
+@pytest.mark.parametrize("fmts", SEARCH_FOUND, ids=lambda f: "p%d.%d.%d_a%d.%d.%d_r%d" % (f[0].as_tuple()[:3] + f[1].as_tuple()[:4]))
+def test_formats_found_by_random_search(fmts):
+    prod, acc = fmts
+    rng = np.random.default_rng(99)
+    finite = np.array([b for b in range(256) if (b & 0x7F) != 0x7F], dtype=np.uint8)
+    for (M, N, K) in ((140, 159, 255), (8, 188, 100)):
+        A = torch.from_numpy(finite[rng.integers(0, finite.size, (M, K))] & 0x7F)             # one sign
+        B = torch.from_numpy(np.where(rng.random((N, K)) < 0.85, 0, finite[rng.integers(0, finite.size, (N, K))]).astype(np.uint8))
+        G = synth.gemm_case(M, N, K, config=77)
+        one = torch.ones(1)
+        for tile in (-1, 0, 3):
+            lba.set_tile_override(tile)
+            try:
+                for order, chunk in ((SEQ, 16), (CHK, 16), (CHK, 32)):
+                    for (a, b) in ((A, B), (G[0], B), (G[0], G[2])):
+                        got = gpu_gemm(a, b, one, one, None, prod, acc, order, chunk)
+                        assert_bit_equal(got, ref_gemm(a, b, one, one, None, prod, acc, order, chunk),
+                                         f"{prod} {acc} {M}x{N}x{K} tile {tile} order {order}/{chunk}")
+            finally:
+                lba.set_tile_override(-1)
+
+
 @pytest.mark.parametrize("tile", [0, 2, 3])
 @pytest.mark.parametrize("name", ["m7e4_code", "m7e4_code_rne", "m4e4_rne", "m10e6_rne", "m7e4_no_uf", "m8e6"])
 def test_slow_climb_to_saturation_crosses_every_clamp_decision(tile, name):
