@@ -39,6 +39,8 @@ def _codes(rng, shape, kind, m4e3):
         c = np.where(rng.random(n) < 0.85, 0, c).astype(np.uint8)
     elif kind == "small":
         c = (c & 0x87) | (rng.integers(0, 3, n, dtype=np.uint8) << 3)   # the lowest binades: products near R_UF
+    elif kind == "climb":
+        c = (c & 0x07) | (rng.integers(3, 9, n, dtype=np.uint8) << 3)   # one sign, middle binades: sums climb slowly to R_OF
     return torch.from_numpy(np.ascontiguousarray(c.reshape(shape)))
 
 
@@ -77,7 +79,7 @@ def _differ(got, want, what):
 
 
 def _one_case(rng, trial):
-    kind = str(rng.choice(["gemm"] * 11 + ["conv"] * 3 + ["fixed"] * 2 + ["batched", "host", "ste", "ste", "last"]))
+    kind = str(rng.choice(["gemm"] * 10 + ["conv"] * 3 + ["fixed"] * 2 + ["batched", "host", "static", "ste", "ste", "last"]))
     prod, acc, m4e3 = _fixed_formats(rng) if kind == "fixed" else _formats(rng)
     if kind in ("ste", "last"):     # floor rounding and E4M3 bytes only
         prod = LbaFormat(prod.man_bits, prod.exp_bits, prod.bias, 0, prod.flags & 1)
@@ -85,11 +87,14 @@ def _one_case(rng, trial):
         m4e3 = False
     small = kind in ("ste", "last", "conv")
     M, N = int(rng.integers(1, 120 if small else 280)), int(rng.integers(1, 120 if small else 280))
-    K = int(rng.choice([0, 1, 2, 15, 16, 17, 31, 33, 64, 100, 255, 256, 500, int(rng.integers(1, 700))]))
+    K = int(rng.choice([0, 1, 2, 15, 16, 17, 31, 33, 64, 100, 255, 256, 500, int(rng.integers(1, 700)), int(rng.integers(1, 700))]))
+    if kind in ("gemm", "fixed", "host") and rng.random() < 0.03:     # a few long chains and wide shapes
+        K = int(rng.choice([1000, 2048, 4100]))
+        M, N = (int(rng.integers(1, 700)), int(rng.integers(1, 130))) if rng.random() < 0.5 else (M, N)
     order = SEQ if (rng.random() < 0.35 or kind == "last") else CHK
     chunk = int(rng.choice([16, 16, 16, 1, 2, 7, 32, 48, 64, int(rng.integers(1, 100))]))
-    tile = int(rng.choice([-1, -1, 0, 1, 2, 3]))
-    ka, kb = rng.choice(["uniform", "gauss", "one_sign", "sparse", "small"], 2)
+    tile = int(rng.choice([-1, -1, -1, 0, 1, 2, 3, 5]))
+    ka, kb = rng.choice(["uniform", "gauss", "one_sign", "sparse", "small", "climb"], 2)
     stride = pad = None
     if kind == "conv":
         Bn, H, W = int(rng.integers(1, 4)), int(rng.integers(1, 16)), int(rng.integers(1, 16))
@@ -128,6 +133,10 @@ def _one_case(rng, trial):
             ws = torch.empty(lba.gemm_host_workspace_bytes(M, N, K, sa.numel(), sb.numel(), bias is not None) + 256,
                              dtype=torch.uint8, device=DEV)
             lba.lba_gemm_host(A, B, sa, sb, bias, prod, acc, order, chunk, got, ws)
+            torch.cuda.synchronize()
+        elif kind == "static":
+            got = torch.empty((M, N), dtype=torch.float32)
+            lba.lba_gemm_host_static(A, B, sa, sb, bias, prod, acc, order, chunk, got)
             torch.cuda.synchronize()
         elif kind == "ste":
             got = lba.lba_gemm_ste_mask(d(A), d(B), prod, acc, order, chunk, *ste)
