@@ -55,7 +55,8 @@ MIX = {
     "rne_wide": (1.0, 0.0, 0.0, 1.0, "1 FFMA (24-bit accumulator: one IEEE FMA per MAC)"),
     "generic": (6.0, 4.0, 0.0, 2.0, "scalar FMUL + FFMA + mask + clamp (+ product steps): the generic kernel"),
     "fixed": (6.0, 4.0, 0.0, 2.0, "2 SHF + 2 add-min/max on the logic pipe; IMAD + IADD beside them"),
-    "ste_diff": (11.0, 5.0, 0.0, 6.0, "FMUL + FFMA + LOP3 + FMNMX + 3 FMUL + 2 FADD + FSETP + bit insert, scalar"),
+    "ste_diff": (7.0, 3.0, 3.0, 1.0, "0.5 each of FMUL2, FFMA2 (chain), FMUL2, FFMA2 (distance), FFMA2, FMUL2 (threshold) "
+                                     "+ LOP3 + FMNMX + FADD (thr - |d|) + SHF (its sign into the mask)"),
 }
 FOLD = {  # per output per chunk: (issue, logic, packed_fp, scalar_fp)
     "floor": (2.5, 2.0, 0.5, 0.0), "rne": (3.5, 2.0, 1.5, 0.0), "rne_wide": (1.0, 0.0, 0.0, 1.0), "generic": (4.0, 2.0, 0.0, 1.0),

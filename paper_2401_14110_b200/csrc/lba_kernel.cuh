@@ -110,6 +110,11 @@ __device__ __forceinline__ float mul_ieee(float a, float b) {  // subnormal oper
   asm("mul.rn.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
   return d;
 }
+__device__ __forceinline__ float add_ieee(float a, float b) {
+  float d;
+  asm("add.rn.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
 __device__ __forceinline__ float fma_rz_ftz(float a, float b, float c) {
   float d;
   asm("fma.rz.ftz.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -197,6 +202,80 @@ __device__ __forceinline__ float decode_m4e3_top(uint32_t top) {
 
 __device__ __forceinline__ uint32_t byte_to_top(uint32_t word, int j) {  // j in 0..3
   return __byte_perm(word, 0u, (uint32_t)(j << 12) | 0x0444u);
+}
+
+// ------------------------------------------------------------------ packed building blocks
+// Two binary32 values in one 64-bit register pair and the f32x2 instructions of sm_100 on them.
+typedef unsigned long long u64;
+
+__device__ __forceinline__ u64 pack2(float lo, float hi) {
+  u64 d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 mul2_ftz(u64 a, u64 b) {
+  u64 d;
+  asm("mul.rn.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ u64 fma2_rz_ftz(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rz.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 fma2_rn(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ u64 fma2_rn_ftz(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rn.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+// Nearest-even cut of a pair of binary32 values to M mantissa bits on the FP32 pipe.  With e the value's own
+// exponent, K = 1.5 * 2^(23-M) * 2^e (same sign) moves the value into a binade whose unit in the last place is the
+// target grid step, so the addition v + K itself rounds to nearest-even on that grid (K/ulp is even, so ties carry
+// over); subtracting K again is exact.  k0 = +-1.5 * 2^e is one logic operation per value (sign and exponent
+// kept, mantissa set to 1.5), and both steps are one packed FMA each: r = k0 * ks + v, result = k0 * (-ks) + r
+// with ks = 2^(23-M).  A zero stays zero (k0 is then a subnormal; r = k0 * ks is cancelled exactly).  Needs M <= 21
+// and exponent headroom for K, which the host checks.  `v` must be exact (or the correctly rounded binary32 image
+// of a sum whose rounding cannot decide an M-bit tie; see the host's conditions for the packed nearest-even path).
+__device__ __forceinline__ u64 rne2_fp(u64 v, u64 ks, u64 nks) {
+  uint32_t lo, hi;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+  u64 k0;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(k0) : "r"((lo & 0xFF800000u) | 0x00400000u), "r"((hi & 0xFF800000u) | 0x00400000u));
+  const u64 r = fma2_rn(k0, ks, v);
+  return fma2_rn(k0, nks, r);
+}
+__device__ __forceinline__ u64 mul2_rn_ftz(u64 a, u64 b) {
+  u64 d;
+  asm("mul.rn.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ u64 add2_rn_ftz(u64 a, u64 b) {
+  u64 d;
+  asm("add.rn.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ u64 mul2_rz_ftz(u64 a, u64 b) {
+  u64 d;
+  asm("mul.rz.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ u64 add2_rz_ftz(u64 a, u64 b) {
+  u64 d;
+  asm("add.rz.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ u64 mul2_rn(u64 a, u64 b) {  // subnormal operands and results honoured
+  u64 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
 }
 
 // ------------------------------------------------------------------ operand fetch
@@ -515,10 +594,55 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), TRACK == TRACK_MASK_DIF
       const float4 v = *reinterpret_cast<const float4*>(&Bs[buf][kk][h * (BN / 2) + tx * 4]);
       b[h * 4 + 0] = v.x; b[h * 4 + 1] = v.y; b[h * 4 + 2] = v.z; b[h * 4 + 3] = v.w;
     }
-    float ad[DIFF ? TM : 1];
-    if (DIFF) {
+    if constexpr (DIFF) {
+      // STE^DIFF: two neighbouring columns share the packed instructions.  Per pair and step: product, sum, the sum
+      // in the comparison's scaling, its distance from the previous one, |x w| + eps1 and the threshold are one f32x2
+      // instruction each; every rounding is the scalar definition's (the products and rescalings are exact).  The bit
+      // is the sign of thr - |d| (negative exactly when |d| > thr: a difference of two binary32 numbers never rounds
+      // to zero), shifted into the slab's halfword from below, so the halfword holds the steps in reverse until the
+      // slab ends.
+      u64 b2[TN / 2], babs2[TN / 2];
 #pragma unroll
-      for (int i = 0; i < TM; ++i) ad[DIFF ? i : 0] = mul_ieee(a[i], p.diff_a_scale);
+      for (int jp = 0; jp < TN / 2; ++jp) {
+        b2[jp] = pack2(b[2 * jp], b[2 * jp + 1]);
+        babs2[jp] = pack2(fabsf(b[2 * jp]), fabsf(b[2 * jp + 1]));
+      }
+      const u64 cc2 = pack2(cc, cc), ds2 = pack2(dscale, dscale), m1 = pack2(-1.0f, -1.0f);
+      const u64 e1 = pack2(deps1, deps1), e2 = pack2(deps2, deps2);
+#pragma unroll
+      for (int i = 0; i < TM; ++i) {
+        const u64 a2 = pack2(a[i], a[i]);
+        const float ada = fabsf(mul_ieee(a[i], p.diff_a_scale));
+        const u64 ada2 = pack2(ada, ada);
+#pragma unroll
+        for (int jp = 0; jp < TN / 2; ++jp) {
+          u64 pr = mul2_ftz(a2, b2[jp]);  // exact; flushes |x w| < R_UF_prod
+          if (QM == QM_FLOOR_FULL) {
+            float plo, phi;
+            unpack2(pr, plo, phi);
+            pr = pack2(clamp_mag(and_bits(plo, qp.mask), qp.sat), clamp_mag(and_bits(phi, qp.mask), qp.sat));
+          }
+          float lo, hi;
+          unpack2(fma2_rz_ftz(pr, cc2, pack2(acc1[i][2 * jp], acc1[i][2 * jp + 1])), lo, hi);
+          lo = clamp_mag(and_bits(lo, qa.mask), qa.sat);
+          hi = clamp_mag(and_bits(hi, qa.mask), qa.sat);
+          acc1[i][2 * jp] = lo;
+          acc1[i][2 * jp + 1] = hi;
+          const u64 zd = mul2_rn(pack2(lo, hi), ds2);                                   // exact: the sums are normal numbers
+          float& p0 = prev1[DIFF ? i : 0][DIFF ? 2 * jp : 0];
+          float& p1 = prev1[DIFF ? i : 0][DIFF ? 2 * jp + 1 : 0];
+          float dlo, dhi, tlo, thi;
+          unpack2(fma2_rn(pack2(p0, p1), m1, zd), dlo, dhi);                            // zd - S_prev, one rounding
+          unpack2(zd, p0, p1);
+          unpack2(mul2_rn(fma2_rn(ada2, babs2[jp], e1), e2), tlo, thi);                 // eps2 * (|x w| + eps1)
+          uint32_t& h0 = half1[MASKS ? i : 0][MASKS ? 2 * jp : 0];
+          uint32_t& h1 = half1[MASKS ? i : 0][MASKS ? 2 * jp + 1 : 0];
+          h0 = __funnelshift_l(__float_as_uint(add_ieee(tlo, -fabsf(dlo))), h0, 1);
+          h1 = __funnelshift_l(__float_as_uint(add_ieee(thi, -fabsf(dhi))), h1, 1);
+        }
+      }
+      (void)kk;
+      return;
     }
 #pragma unroll
     for (int i = 0; i < TM; ++i)
@@ -533,7 +657,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), TRACK == TRACK_MASK_DIF
           if (LAST) {
             if (fabsf(t) >= qa.sat && real_step) last[LAST ? i : 0][LAST ? j : 0] = kbase + kk;
           } else {
-            const float u = DIFF ? mul_ieee(ad[DIFF ? i : 0], b[j]) : 0.0f;  // exact |x w| in the comparison's scaling
+            const float u = 0.0f;
             // bit kk of the slab's halfword; steps past K are cleared when the halfword joins its word
             if (ste_bit(t, z, u, prev1[DIFF ? i : 0][DIFF ? j : 0])) half1[MASKS ? i : 0][MASKS ? j : 0] |= 1u << kk;
           }
@@ -556,8 +680,10 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), TRACK == TRACK_MASK_DIF
   for (int s = 0; s < nslab; ++s) {
     const int buf = s & 1;
     if (s + 1 < nslab) fetch(s + 1, raw);
+    int steps_run = BK;  // mac_step calls of this slab
     if (ORD == ORD_CHUNK_ANY) {
       const int kmax = (int)((K - (int64_t)s * BK) < BK ? (K - (int64_t)s * BK) : BK);
+      steps_run = kmax;
 #pragma unroll 1
       for (int kk = 0; kk < kmax; ++kk) {
         mac_step(buf, kk);
@@ -584,6 +710,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), TRACK == TRACK_MASK_DIF
       for (int i = 0; i < TM; ++i)
 #pragma unroll
         for (int j = 0; j < TN; ++j) {
+          // STE^DIFF shifted its bits in from below: step 0 of the slab's `steps_run` steps sits highest
+          if (DIFF) half1[i][j] = steps_run > 0 ? (__brev(half1[i][j]) >> (32 - steps_run)) : 0u;
           bits1[i][j] |= (half1[i][j] & keep) << sh;
           half1[i][j] = 0u;
         }
@@ -674,73 +802,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), TRACK == TRACK_MASK_DIF
 // B-row norms of the slab give one bound per CTA, and each thread carries an upper bound `u` of
 // its own |S| (as a fraction of 2^(e_max+1)), refreshed from the registers when it gets too loose.
 // A warp whose bound fails runs the same slab with the clamp.  Results are identical either way.
-typedef unsigned long long u64;
 constexpr int KUNROLL = 16;  // k-steps unrolled in the packed slab body (the whole slab: measured fastest)
 
-__device__ __forceinline__ u64 pack2(float lo, float hi) {
-  u64 d;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
-  return d;
-}
-__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ u64 mul2_ftz(u64 a, u64 b) {
-  u64 d;
-  asm("mul.rn.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-__device__ __forceinline__ u64 fma2_rz_ftz(u64 a, u64 b, u64 c) {
-  u64 d;
-  asm("fma.rz.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ u64 fma2_rn(u64 a, u64 b, u64 c) {
-  u64 d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ u64 fma2_rn_ftz(u64 a, u64 b, u64 c) {
-  u64 d;
-  asm("fma.rn.ftz.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-// Nearest-even cut of a pair of binary32 values to M mantissa bits on the FP32 pipe.  With e the value's own
-// exponent, K = 1.5 * 2^(23-M) * 2^e (same sign) moves the value into a binade whose unit in the last place is the
-// target grid step, so the addition v + K itself rounds to nearest-even on that grid (K/ulp is even, so ties carry
-// over); subtracting K again is exact.  k0 = +-1.5 * 2^e is one logic operation per value (sign and exponent
-// kept, mantissa set to 1.5), and both steps are one packed FMA each: r = k0 * ks + v, result = k0 * (-ks) + r
-// with ks = 2^(23-M).  A zero stays zero (k0 is then a subnormal; r = k0 * ks is cancelled exactly).  Needs M <= 21
-// and exponent headroom for K, which the host checks.  `v` must be exact (or the correctly rounded binary32 image
-// of a sum whose rounding cannot decide an M-bit tie; see the host's conditions for the packed nearest-even path).
-__device__ __forceinline__ u64 rne2_fp(u64 v, u64 ks, u64 nks) {
-  uint32_t lo, hi;
-  asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
-  u64 k0;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(k0) : "r"((lo & 0xFF800000u) | 0x00400000u), "r"((hi & 0xFF800000u) | 0x00400000u));
-  const u64 r = fma2_rn(k0, ks, v);
-  return fma2_rn(k0, nks, r);
-}
-__device__ __forceinline__ u64 mul2_rn_ftz(u64 a, u64 b) {
-  u64 d;
-  asm("mul.rn.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-__device__ __forceinline__ u64 add2_rn_ftz(u64 a, u64 b) {
-  u64 d;
-  asm("add.rn.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-__device__ __forceinline__ u64 mul2_rz_ftz(u64 a, u64 b) {
-  u64 d;
-  asm("mul.rz.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-__device__ __forceinline__ u64 add2_rz_ftz(u64 a, u64 b) {
-  u64 d;
-  asm("add.rz.ftz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
 // two E4M3 bytes (low 16 bits of `pair`) -> their exact values, by the hardware converter
 __device__ __forceinline__ void e4m3x2_to_f32(uint32_t pair, float& v0, float& v1) {
   asm("{\n\t.reg .b16 c, lo, hi;\n\t.reg .b32 h;\n\t"
