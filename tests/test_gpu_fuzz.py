@@ -96,6 +96,7 @@ def _one_case(rng, trial):
     tile = int(rng.choice([-1, -1, -1, 0, 1, 2, 3, 5]))
     ka, kb = rng.choice(["uniform", "gauss", "one_sign", "sparse", "small", "climb"], 2)
     stride = pad = None
+    misaligned = bool(rng.random() < 0.15)
     if kind == "conv":
         Bn, H, W = int(rng.integers(1, 4)), int(rng.integers(1, 16)), int(rng.integers(1, 16))
         Cin = int(rng.choice([1, 3, 4, 5, 16, 24, 32, 48, 64]))
@@ -143,7 +144,11 @@ def _one_case(rng, trial):
         elif kind == "last":
             got = lba.lba_gemm_last_overflow(d(A), d(B), prod, acc)
         else:
-            got = lba.lba_gemm(d(A), d(B), d(sa), d(sb), d(bias), prod, acc, order, chunk)
+            # now and then from operands and into an output that start off a 16-byte boundary (the byte-wise loader, scalar stores)
+            shift = lambda t, o: torch.cat([t.new_zeros(o), t.reshape(-1)])[o:].view(t.shape)
+            oa, ob, oo = (int(v) for v in rng.integers(0, 16, 3)) if misaligned else (0, 0, 0)
+            out = shift(torch.empty((M, N), dtype=torch.float32, device=DEV), oo % 4)
+            got = lba.lba_gemm(shift(d(A), oa), shift(d(B), ob), d(sa), d(sb), d(bias), prod, acc, order, chunk, out=out)
     except lba.LbaError as e:
         assert e.status == ERR_FORMAT, what + f": {e}"
         return False
