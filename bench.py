@@ -434,6 +434,26 @@ def other_configs(device, sm_count, max_mhz, headline_wl):
     ms, per = time_workload(wl, 200, 20)
     e = summary_entry(wl, ms, per, sm_count, max_mhz)
     e["us_per_launch"] = per[0] * 1e3
+    # the same launch replayed from a CUDA graph (32 per replay): the device time without the host's launch path
+    side = torch.cuda.Stream(device=device)
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        wl.run_step()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for _ in range(32):
+            wl.run_step()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(3):
+        graph.replay()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(10):
+        graph.replay()
+    t1.record()
+    torch.cuda.synchronize()
+    e["us_per_launch_in_graph"] = t0.elapsed_time(t1) * 1e3 / 320
+    e["gmacs_in_graph"] = wl.macs / (e["us_per_launch_in_graph"] * 1e-6) / 1e9
     e["note"] = "latency-bound by construction: 4096 outputs, 576 dependent steps each"
     out["config1_gemm_64x64x576_sequential"] = e
     # configs 2 and 3: the convolution stacks

@@ -29,7 +29,10 @@
  * memory, keeps no state between calls except the last CUDA error code (and the testing hook
  * lba_set_tile_override), and never
  * synchronises: work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default
- * stream).  Format structs are read on the host during the call.
+ * stream).  Format structs are read on the host during the call.  Because a call only enqueues
+ * kernels (and, in the host-buffer variants, asynchronous copies), it may be recorded by a stream
+ * capture and replayed from a CUDA graph; the recorded launch shape is the one chosen for the
+ * sizes and formats given at capture time.
  *
  * Preconditions that are not checked on the device: no input byte is an E4M3 NaN code
  * (0x7F, 0xFF; use lba_count_nan_codes to check), scales are finite and > 0.  Every zero

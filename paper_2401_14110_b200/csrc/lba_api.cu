@@ -80,6 +80,8 @@ struct Plan {
   int chunk_slabs, chunk;
   int kp, ka, sx;   // product carrier = value * 2^kp, accumulator carrier = value * 2^ka, A operand = x * 2^sx
   int in_m4e3;      // operands are M4E3 bytes
+  int sum_grid;     // every sum is a multiple of 2^sum_grid
+  bool a_flush;     // the flush of Q_acc is reachable
   int fused;        // Q_prod is the identity on every reachable product: PQ_FUSED applies (plain packed tiles)
   float pk_b_fused; // B operand scaling for it: 2^(sw + ka - kp), so that x' w' lands in the accumulator carrier
   double a_top;     // largest reachable accumulator magnitude (real domain)
@@ -198,6 +200,8 @@ int make_plan(const lba_fmt* pf, const lba_fmt* af, int order, int chunk, int64_
   // carrier places that step at the smallest normal number
   const bool a_flush = (af->flags & LBA_FLAG_UNDERFLOW) && -af->bias > sum_grid;
   const int ka = a_flush ? af->bias - 126 : -126 - sum_grid;
+  pl->sum_grid = sum_grid;
+  pl->a_flush = a_flush;
   float a_sat_carrier = FLT_MAX;
   if (a_sat) {
     if (a_emax + ka < -126 || a_emax + ka > 127) return LBA_ERR_FORMAT;
@@ -630,9 +634,9 @@ int lba_gemm_ste_mask(const uint8_t* A, const uint8_t* B, int64_t M, int64_t N, 
     };
     const double u_max = std::fmax(std::ldexp(1.0, 18), pl.a_top);   // |x w| < 2^18; a chunk sum <= a_top
     const double u_min = std::ldexp(1.0, -18);                       // smallest non-zero |x w| and chunk sum
-    // smallest non-zero |z - S|: one step of the accumulator's grid in its lowest binade
-    const bool a_flush = (acc_fmt->flags & LBA_FLAG_UNDERFLOW) && acc_fmt->bias < 18;
-    const double d_min = a_flush ? std::ldexp(1.0, -acc_fmt->bias - acc_fmt->man_bits) : u_min;
+    // smallest non-zero |z - S|: one step of the accumulator's grid in its lowest binade where sums below R_UF are
+    // flushed, else one step of the grid on which every sum lies
+    const double d_min = pl.a_flush ? std::ldexp(1.0, -acc_fmt->bias - acc_fmt->man_bits) : std::ldexp(1.0, pl.sum_grid);
     for (const double v : {(double)eps1, u_max + eps1, (double)eps2 * eps1, (double)eps2 * (u_max + eps1), u_min, u_max,
                            d_min, 2.0 * pl.a_top})
       if (!normal(v)) return LBA_ERR_FORMAT;

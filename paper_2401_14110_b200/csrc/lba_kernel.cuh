@@ -597,7 +597,8 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), TRACK == TRACK_MASK_DIF
     if constexpr (DIFF) {
       // STE^DIFF: two neighbouring columns share the packed instructions.  Per pair and step: product, sum, the sum
       // in the comparison's scaling, its distance from the previous one, |x w| + eps1 and the threshold are one f32x2
-      // instruction each; every rounding is the scalar definition's (the products and rescalings are exact).  The bit
+      // instruction each; every rounding is the scalar definition's (the products and rescalings are exact; the previous
+      // sum of the first hierarchy is the accumulator itself before the step, so only the folds keep a copy).  The bit
       // is the sign of thr - |d| (negative exactly when |d| > thr: a difference of two binary32 numbers never rounds
       // to zero), shifted into the slab's halfword from below, so the halfword holds the steps in reverse until the
       // slab ends.
@@ -607,7 +608,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), TRACK == TRACK_MASK_DIF
         b2[jp] = pack2(b[2 * jp], b[2 * jp + 1]);
         babs2[jp] = pack2(fabsf(b[2 * jp]), fabsf(b[2 * jp + 1]));
       }
-      const u64 cc2 = pack2(cc, cc), ds2 = pack2(dscale, dscale), m1 = pack2(-1.0f, -1.0f);
+      const u64 cc2 = pack2(cc, cc), ds2 = pack2(dscale, dscale), nds2 = pack2(-dscale, -dscale);
       const u64 e1 = pack2(deps1, deps1), e2 = pack2(deps2, deps2);
 #pragma unroll
       for (int i = 0; i < TM; ++i) {
@@ -623,17 +624,15 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN), TRACK == TRACK_MASK_DIF
             pr = pack2(clamp_mag(and_bits(plo, qp.mask), qp.sat), clamp_mag(and_bits(phi, qp.mask), qp.sat));
           }
           float lo, hi;
-          unpack2(fma2_rz_ftz(pr, cc2, pack2(acc1[i][2 * jp], acc1[i][2 * jp + 1])), lo, hi);
+          const u64 s_old = pack2(acc1[i][2 * jp], acc1[i][2 * jp + 1]);
+          unpack2(fma2_rz_ftz(pr, cc2, s_old), lo, hi);
           lo = clamp_mag(and_bits(lo, qa.mask), qa.sat);
           hi = clamp_mag(and_bits(hi, qa.mask), qa.sat);
           acc1[i][2 * jp] = lo;
           acc1[i][2 * jp + 1] = hi;
           const u64 zd = mul2_rn(pack2(lo, hi), ds2);                                   // exact: the sums are normal numbers
-          float& p0 = prev1[DIFF ? i : 0][DIFF ? 2 * jp : 0];
-          float& p1 = prev1[DIFF ? i : 0][DIFF ? 2 * jp + 1 : 0];
           float dlo, dhi, tlo, thi;
-          unpack2(fma2_rn(pack2(p0, p1), m1, zd), dlo, dhi);                            // zd - S_prev, one rounding
-          unpack2(zd, p0, p1);
+          unpack2(fma2_rn(s_old, nds2, zd), dlo, dhi);          // zd - S_prev * dscale (exact product), one rounding
           unpack2(mul2_rn(fma2_rn(ada2, babs2[jp], e1), e2), tlo, thi);                 // eps2 * (|x w| + eps1)
           uint32_t& h0 = half1[MASKS ? i : 0][MASKS ? 2 * jp : 0];
           uint32_t& h1 = half1[MASKS ? i : 0][MASKS ? 2 * jp + 1 : 0];

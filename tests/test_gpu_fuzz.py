@@ -20,6 +20,7 @@ DEV = "cuda:0"
 CASES = int(os.environ.get("LBA_FUZZ_CASES", "400"))
 SEED = int(os.environ.get("LBA_FUZZ_SEED", "20240125"))
 ERR_FORMAT = -3
+UNCHECKED = []   # cases the library ran and the oracle could not carry
 
 
 def _codes(rng, shape, kind, m4e3):
@@ -54,10 +55,11 @@ def _formats(rng):
         bp = 2 ** E - (16 if m4e3 else 18) + int(rng.integers(-3, 4))
         prod = LbaFormat(M, E, bp, rounding, flags | (FLAG_INPUT_M4E3 if m4e3 else 0))
         acc = LbaFormat(int(rng.choice([M, M, max(1, M - 2), min(23, M + 3)])), E, bp - int(rng.integers(0, 5)), rounding, flags)
-    else:                        # anything the header admits
-        prod = LbaFormat(int(rng.integers(1, 24)), int(rng.integers(1, 9)), int(rng.integers(-20, 40)), rounding,
+    else:                        # anything the header admits (the far ends of the bias range now and then)
+        lo, hi = (-96, 193) if rng.random() < 0.2 else (-20, 40)
+        prod = LbaFormat(int(rng.integers(1, 24)), int(rng.integers(1, 9)), int(rng.integers(lo, hi)), rounding,
                          flags | (FLAG_INPUT_M4E3 if m4e3 else 0))
-        acc = LbaFormat(int(rng.integers(1, 24)), int(rng.integers(1, 9)), int(rng.integers(-20, 40)), rounding, flags)
+        acc = LbaFormat(int(rng.integers(1, 24)), int(rng.integers(1, 9)), int(rng.integers(lo, hi)), rounding, flags)
     return prod, acc, m4e3
 
 
@@ -154,6 +156,16 @@ def _one_case(rng, trial):
         return False
     finally:
         lba.set_tile_override(-1)
+    try:
+        _compare(kind, got, A, B, sa, sb, bias, stride, pad, pt, at, order, chunk, ste, what)
+    except orc.OracleError:   # the span of the operands exceeds the oracle's exact 126-bit carrier: the case cannot be checked
+        UNCHECKED.append(what)
+        return False
+    return True
+
+
+def _compare(kind, got, A, B, sa, sb, bias, stride, pad, pt, at, order, chunk, ste, what):
+    n = lambda t: None if t is None else t.numpy()
     if kind == "conv":
         _differ(got.cpu().numpy(), orc.conv2d(n(A), n(B), n(sa), n(sb), n(bias), stride, pad, pt, at, order, chunk), what)
     elif kind == "batched":
@@ -171,7 +183,6 @@ def _one_case(rng, trial):
         _differ(got.cpu().numpy(), orc.gemm_last_overflow(n(A), n(B), pt, at), what)
     else:
         _differ(got.cpu().numpy(), orc.gemm(n(A), n(B), n(sa), n(sb), n(bias), pt, at, order, chunk), what)
-    return True
 
 
 def test_random_formats_shapes_and_operands():
@@ -180,3 +191,4 @@ def test_random_formats_shapes_and_operands():
     # formats the library declines (a carrier out of binary32's range, 22 mantissa bits with nearest-even, ...) are
     # declined with the format status; most draws must run
     assert ran >= CASES // 2, f"only {ran} of {CASES} random cases were accepted"
+    assert len(UNCHECKED) <= CASES // 50, f"{len(UNCHECKED)} cases could not be checked, e.g. {UNCHECKED[0]}"

@@ -804,3 +804,35 @@ def test_nan_code_counter():
     codes[17] = 0x7F
     codes[99999] = 0xFF
     assert lba.count_nan_codes(codes.to(DEV)) == 2
+
+
+def test_calls_are_capturable_in_a_cuda_graph():
+    # the entry points only enqueue work on the given stream (no allocation, no synchronisation), so a stream capture
+    # records them; the replayed graph gives the oracle's bits for GEMM and convolution alike, on fresh operands too
+    prod, acc = code_domain_formats(7, 4)
+    A, sa, B, sb = synth.gemm_case(70, 45, 100, config=3)
+    dA, dB, dsa, dsb = A.to(DEV), B.to(DEV), sa.to(DEV), sb.to(DEV)
+    out = torch.zeros((70, 45), dtype=torch.float32, device=DEV)
+    x = synth.random_codes((2, 9, 9, 16), 30).to(DEV)
+    w = synth.random_codes((40, 3, 3, 16), 31).to(DEV)
+    one = torch.ones(1, device=DEV)
+    cout = torch.zeros((2, 9, 9, 40), dtype=torch.float32, device=DEV)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):   # first use outside the capture (function attributes are set once per kernel)
+        lba.lba_gemm(dA, dB, dsa, dsb, None, prod, acc, CHK, 16, out=out)
+        lba.lba_conv2d(x, w, one, one, None, (1, 1), (1, 1), prod, acc, CHK, 16, out=cout)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        lba.lba_gemm(dA, dB, dsa, dsb, None, prod, acc, CHK, 16, out=out)
+        lba.lba_conv2d(x, w, one, one, None, (1, 1), (1, 1), prod, acc, CHK, 16, out=cout)
+    torch.cuda.current_stream().wait_stream(side)
+    A2 = synth.random_codes((70, 100), 77)
+    dA.copy_(A2.to(DEV))
+    out.zero_()
+    cout.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert_bit_equal(out, ref_gemm(A2, B, sa, sb, None, prod, acc, CHK, 16), "graph replay, GEMM")
+    want = orc.conv2d(x.cpu().numpy(), w.cpu().numpy(), 1.0, 1.0, None, (1, 1), (1, 1), prod.as_tuple(), acc.as_tuple(), CHK, 16)
+    assert_bit_equal(cout, want, "graph replay, convolution")
