@@ -1010,7 +1010,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
         // floor: the products of micro-tile row i + 1 are formed while row i is added and masked, so that
         // multiplies (FP32 pipe) and masks (logic pipe) of independent outputs sit side by side in the stream
         auto product = [&](u64 av, u64 bv) -> u64 {
-          u64 pr = mul2_ftz(av, bv);
+          u64 pr = mul2_ftz(bv, av);
           if (PQ == PQ_MASK || PQ == PQ_MASK_SAT) {  // floor of Eq. 2 on the exact product, then its saturation
             float plo, phi;
             unpack2(pr, plo, phi);
@@ -1029,7 +1029,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
           for (int i = 0; i < TM; ++i)
 #pragma unroll
             for (int j = 0; j < PN; ++j) {
-              const u64 t = (CH16 && kk == 0) ? mul2_rz_ftz(a2[i], b2[j]) : fma2_rz_ftz(a2[i], b2[j], acc1[i][j]);
+              const u64 t = (CH16 && kk == 0) ? mul2_rz_ftz(b2[j], a2[i]) : fma2_rz_ftz(b2[j], a2[i], acc1[i][j]);
               float lo, hi;
               unpack2(t, lo, hi);
               lo = and_bits(lo, mask);
@@ -1057,7 +1057,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
           }
 #pragma unroll
           for (int j = 0; j < PN; ++j) {
-            const u64 t = (CH16 && kk == 0) ? mul2_rz_ftz(pr[j], cc2) : fma2_rz_ftz(pr[j], cc2, acc1[i][j]);
+            const u64 t = (CH16 && kk == 0) ? mul2_rz_ftz(cc2, pr[j]) : fma2_rz_ftz(cc2, pr[j], acc1[i][j]);
             float lo, hi;
             unpack2(t, lo, hi);
             lo = and_bits(lo, mask);
@@ -1091,9 +1091,9 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
           // `.ftz` flushes exactly the sums below R_UF_acc: such a sum is a short dyadic number and survives as a subnormal.
           u64 v;
           if constexpr (PQ == PQ_FUSED) {  // Q_prod is the identity: product and sum in one FMA
-            v = (CH16 && kk == 0) ? mul2_rn_ftz(a2[i], b2[j]) : fma2_rn_ftz(a2[i], b2[j], acc1[i][j]);
+            v = (CH16 && kk == 0) ? mul2_rn_ftz(b2[j], a2[i]) : fma2_rn_ftz(b2[j], a2[i], acc1[i][j]);
           } else {
-            u64 pr = mul2_ftz(a2[i], b2[j]);
+            u64 pr = mul2_ftz(b2[j], a2[i]);
             if (PQ == PQ_MASK || PQ == PQ_MASK_SAT) {  // nearest-even on the exact product, then its saturation
               pr = rne2_fp(pr, ks_prod, nks_prod);
               if (PQ == PQ_MASK_SAT) {
@@ -1102,7 +1102,7 @@ __global__ void __launch_bounds__((BM / TM) * (BN / TN),
                 pr = pack2(clamp_mag(plo, psat), clamp_mag(phi, psat));
               }
             }
-            v = (CH16 && kk == 0) ? mul2_rn_ftz(pr, cc2) : fma2_rn_ftz(pr, cc2, acc1[i][j]);
+            v = (CH16 && kk == 0) ? mul2_rn_ftz(cc2, pr) : fma2_rn_ftz(cc2, pr, acc1[i][j]);
           }
           float lo, hi;
           const u64 q = rne2_fp(v, ks_acc, nks_acc);
