@@ -116,22 +116,22 @@ def peak_gmacs(mode, chunk, sm_count, mhz):
 
 # DRAM bytes (read + write) of ONE launch of the dominant kernel, from the ncu captures summarised under profiles/
 # (workload, kernel description) -> (bytes, what was captured, executed instructions per emulated MAC).
-_K_FLOOR = "tile=64x64x16 micro=4x8 q=floor_fast pq=none kernel=packed order=chunk16 load=gemm_vec"
+_K_FLOOR = "tile=128x128x16 micro=8x8 q=floor_fast pq=none kernel=packed order=chunk16 load=gemm_vec"
 _CAP = "profiles/packed_floor_kernel_gemm_8192x8192x1024_chunk.txt"
 NCU = {
     # the headline launch is too long for a multi-pass capture (52 ms, 39 passes): the K = 1024 case of the same kernel was
     # captured; its reads grow in proportion to K (x 8), its writes (the output) do not grow with K
     ("single_lba_gemm_8192x8192x8192_m7e4_chunk16", _K_FLOOR):
-        (8 * 17442560 + 213800960, "scaled from the 8192x8192x1024 capture (" + _CAP + "): 8 x 17.4 MB read + 213.8 MB written; "
-         "algorithmic 128 MB + 256 MB (part of the output is still in L2 when the kernel ends)", 2.630),
+        (8 * 17673984 + 214364672, "scaled from the 8192x8192x1024 capture (" + _CAP + "): 8 x 17.7 MB read + 214.4 MB written; "
+         "algorithmic 128 MB + 256 MB (part of the output is still in L2 when the kernel ends)", 2.453),
     ("single_lba_gemm_8192x8192x1024_m7e4_chunk16", _K_FLOOR):
-        (17442560 + 213800960, "17.4 MB read + 213.8 MB written (" + _CAP + "); algorithmic 272 MB", 2.630),
+        (17673984 + 214364672, "17.7 MB read + 214.4 MB written (" + _CAP + "); algorithmic 272 MB", 2.453),
     ("single_lba_gemm_8192x8192x1024_m7e4_sequential", "tile=128x128x16 micro=8x8 q=floor_fast pq=none kernel=packed order=seq load=gemm_vec"):
         (18133504 + 212325376, "18.1 MB read + 212.3 MB written (profiles/packed_floor_kernel_gemm_8192x8192x1024_seq.txt)", 2.323),
     ("single_lba_gemm_8192x8192x1024_m7e4_rne_chunk16", "tile=64x64x16 micro=4x8 q=rne_full pq=none kernel=packed order=chunk16 load=gemm_vec"):
         (17937920 + 212977664, "17.9 MB read + 213.0 MB written (profiles/packed_nearest_even_kernel_gemm_8192x8192x1024_chunk.txt)", 4.921),
-    ("single_lba_gemm_8192x8192x1024_m8e6_chunk16", "tile=64x64x16 micro=4x8 q=floor_fast pq=fused kernel=packed order=chunk16 load=gemm_vec"):
-        (16979200 + 213186048, "17.0 MB read + 213.2 MB written (profiles/packed_floor_kernel_fused_gemm_8192x8192x1024_chunk.txt)", 2.128),
+    ("single_lba_gemm_8192x8192x1024_m8e6_chunk16", "tile=128x128x16 micro=8x8 q=floor_fast pq=fused kernel=packed order=chunk16 load=gemm_vec"):
+        (17225472 + 213304832, "17.2 MB read + 213.3 MB written (profiles/packed_floor_kernel_fused_gemm_8192x8192x1024_chunk.txt)", 1.946),
 }
 
 

@@ -344,18 +344,22 @@ int sm_count() {
 // Pick the cheapest by that model.
 // pair_ok: the call qualifies for the 64x64 tile shared by a cluster of two CTAs (TILE_PAIR)
 int choose_tile(int64_t M, int64_t N, int64_t batch, int qm, int ord, int load, bool pair_ok = false) {
-  (void)qm;
   const int forced = g_tile_override.load(std::memory_order_relaxed);
   if (forced >= 0 && forced < TILE_COUNT) return forced;
   if (forced == TILE_PAIR && pair_ok) return TILE_PAIR;
   const int sms = sm_count();
   // relative MAC rate of each tile with every SM loaded (8192^2 x 1024 and 4096 x 3072 x 768 GEMMs)
-  const double eff_seq[TILE_COUNT] = {1.00, 0.91, 0.95, 0.84};
-  const double eff_chunk[TILE_COUNT] = {0.97, 0.96, 1.00, 0.89};
+  const double eff_seq[TILE_COUNT] = {1.00, 0.92, 0.96, 0.82};
+  const double eff_chunk[TILE_COUNT] = {1.00, 0.96, 0.99, 0.87};
+  // nearest-even: three more packed instructions per pair and step; the 8x8 micro-tile loses its lead
+  const double eff_rne_seq[TILE_COUNT] = {1.00, 0.97, 0.99, 0.95};
+  const double eff_rne_chunk[TILE_COUNT] = {0.88, 0.95, 1.00, 0.91};
   // byte-wise loader (ResNet stem, 401408 x 64 x 147): the fetch is costly, so the tile with the fewest
   // fetched rows per output wins as long as it keeps its registers
   const double eff_any[TILE_COUNT] = {0.55, 1.00, 0.87, 0.73};
-  const double* eff = load == LD_ANY ? eff_any : (ord == ORD_SEQ ? eff_seq : eff_chunk);
+  const bool rne = qm == QM_RNE_FULL;
+  const double* eff = load == LD_ANY ? eff_any
+                                     : (ord == ORD_SEQ ? (rne ? eff_rne_seq : eff_seq) : (rne ? eff_rne_chunk : eff_chunk));
   int best = 0;
   double best_cost = 1e300;
   for (int t = 0; t < TILE_COUNT; ++t) {
