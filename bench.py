@@ -154,9 +154,9 @@ def parse_args(argv=None):
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-streams", type=int, default=12,
                     help="network workloads: streams (each with its own device workspace) the end-to-end calls are spread over")
-    ap.add_argument("--e2e-row-blocks", type=int, default=8,
+    ap.add_argument("--e2e-row-blocks", type=int, default=2,
                     help="single-GEMM workloads: the end-to-end step is issued as this many row blocks (rows of the output are "
-                         "independent chains), one lba_gemm_host call each, over three streams, so that one block's copies "
+                         "independent chains), one lba_gemm_host call each, over up to three streams, so that one block's copies "
                          "overlap another block's kernel; 1 = one call")
     ap.add_argument("--force-dist", action="store_true",
                     help="initialise torch.distributed (NCCL) even for a single rank: exercises the multi-GPU plumbing "
