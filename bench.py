@@ -307,13 +307,15 @@ def gemm_operands(m, n, k, device, config=5, outliers=False, weight_std=1.0):
 def build_workload(spec: str, device):
     """A Workload from a --workload string."""
     from paper_2401_14110_b200 import (binding as lba, synth, workloads, code_domain_formats, fixed_point_format,
-                                       ORDER_CHUNKED, ORDER_SEQUENTIAL)
+                                       m4e3_input_formats, ORDER_CHUNKED, ORDER_SEQUENTIAL)
     parts = spec.lower().split(":")
     kind = parts[0]
+    m4e3 = "wa=m4e3" in parts[1:]   # operands in the paper's own weight/activation byte format (Sec. 3.1) instead of OCP E4M3
     if kind in ("resnet18", "resnet50"):
-        prod, acc = code_domain_formats(7, 4)
+        prod, acc = m4e3_input_formats(7, 4) if m4e3 else code_domain_formats(7, 4)
         batch, config = (32, 2) if kind == "resnet18" else (64, 3)
-        wl = Workload(f"{kind}_fwd_conv_stack_b{batch}_224_m7e4_chunk16", prod, acc, ORDER_CHUNKED, batch=batch)
+        wl = Workload(f"{kind}_fwd_conv_stack_b{batch}_224_{'wa_m4e3_' if m4e3 else ''}m7e4_chunk16", prod, acc, ORDER_CHUNKED,
+                      batch=batch)
 
         def conv_fn(x, w, sx, sw, stride, pad):
             return lba.lba_conv2d(x, w, sx, sw, None, stride, pad, prod, acc, ORDER_CHUNKED, 16)
@@ -321,7 +323,8 @@ def build_workload(spec: str, device):
         def gemm_fn(a, b, sa, sb):
             return lba.lba_gemm(a, b, sa, sb, None, prod, acc, ORDER_CHUNKED, 16)
 
-        wl.calls, _ = workloads.build_resnet_calls(kind, batch, config, device, conv_fn, gemm_fn)
+        wl.calls, _ = workloads.build_resnet_calls(kind, batch, config, device, conv_fn, gemm_fn,
+                                                   wa_format="m4e3" if m4e3 else "e4m3")
         return wl.finish(device)
     if kind == "bert":
         seq = "seq" in parts[1:]
@@ -352,8 +355,13 @@ def build_workload(spec: str, device):
     a, sa, b, sb = gemm_operands(m, n, k, device)
     if kind == "gemm":
         M_, E_, rnd = parse_format_tokens(parts[2:])
-        prod, acc = code_domain_formats(M_, E_, rnd)
-        wl = Workload("single_lba_gemm_%dx%dx%d_m%de%d%s_%s" % (m, n, k, M_, E_, "_rne" if rnd else "", oname), prod, acc, order)
+        prod, acc = (m4e3_input_formats if m4e3 else code_domain_formats)(M_, E_, rnd)
+        if m4e3:   # the same Gaussian operands, quantised per tensor to the paper's byte format
+            ga, gb = synth.gaussian((m, k), synth.seed_for(5, 0)), synth.gaussian((n, k), synth.seed_for(5, 1))
+            (a, sa), (b, sb) = synth.quantise_m4e3_per_tensor(ga), synth.quantise_m4e3_per_tensor(gb)
+            a, sa, b, sb = a.to(device), sa.to(device), b.to(device), sb.to(device)
+        wl = Workload("single_lba_gemm_%dx%dx%d_%sm%de%d%s_%s" % (m, n, k, "wa_m4e3_" if m4e3 else "", M_, E_,
+                                                                  "_rne" if rnd else "", oname), prod, acc, order)
         wl.calls = [workloads.LbaCall("gemm", "gemm", a, b, sa, sb)]
     elif kind == "fixed":
         wrap = "wrap" in parts[2:]
