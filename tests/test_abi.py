@@ -99,3 +99,18 @@ def test_host_variants_refuse_shapes_whose_byte_counts_would_wrap():
     # convolution: the output byte count is guarded the same way
     assert lib.lba_conv2d_host_workspace_bytes(1 << 20, 1, 1, 1, 1 << 20, 1, 1, 1, 1, 0, 0, 1, 1, 0) > 0
     assert lib.lba_conv2d_host_workspace_bytes(1 << 30, 1, 1, 1, 1 << 30, 1, 1, 1, 1, 0, 0, 1, 1, 0) == 0     # 4*M*C_out = 2^62
+
+
+def test_tile_choice_follows_the_measured_order():
+    # the host's tile model is fitted to measurements on B200 (148 SMs is also what the model assumes without a device):
+    # these are the shapes it was fitted and checked on, with the tile that measured fastest
+    f, r = code_domain_formats(7, 4), code_domain_formats(7, 4, rounding=1)
+    tile = lambda shape, fm, order: lba.describe_plan(*shape, *fm, order, 16).split(" q=")[0]
+    assert tile((8192, 8192, 8192), f, CHK) == "tile=128x128x16 micro=8x8"       # full SMs, floor: the 8x8 micro-tile
+    assert tile((8192, 8192, 8192), f, SEQ) == "tile=128x128x16 micro=8x8"
+    assert tile((8192, 8192, 8192), r, CHK) == "tile=64x64x16 micro=4x8"         # nearest-even, chunk 16: 64x64 is 12 % faster
+    assert tile((4096, 768, 768), f, CHK) == "tile=64x64x16 micro=4x8"           # BERT linears: not the 32x32 tile
+    assert tile((25088, 128, 1152), f, CHK) == "tile=64x64x16 micro=4x8"         # ResNet-18 layer2
+    assert tile((1568, 512, 4608), f, CHK) == "tile=64x64x16 pair micro=4x8"     # layer4: two CTAs per tile
+    assert tile((1568, 512, 4608), f, SEQ) == "tile=32x32x16 micro=4x4"          # no chunks to share in sequential order
+    assert tile((32, 1000, 512), f, CHK) == "tile=32x32x16 micro=4x4"            # the classifier
