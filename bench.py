@@ -267,7 +267,8 @@ class Workload:
             return "ste_mask=%s tile=64x64x16 micro=%s q=floor order=%s" % (
                 self.ste, "4x8 packed" if self.ste == "of" else "4x4 scalar", "chunk16" if self.order else "seq")
         vec = (c.x.shape[-1] % 16 == 0) if c.kind == "conv" else (k % 16 == 0)
-        return lba.describe_plan(m, n, k, self.prod, self.acc, self.order, self.chunk, is_conv=c.kind == "conv", vec_ok=vec)
+        return lba.describe_plan(m, n, k, self.prod, self.acc, self.order, self.chunk, is_conv=c.kind == "conv", vec_ok=vec,
+                                 batch=c.x.shape[0] if c.kind == "bgemm" else 1)
 
     @property
     def macs(self):

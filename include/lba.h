@@ -245,6 +245,11 @@ int lba_count_nan_codes(const uint8_t* codes, int64_t n, unsigned long long* cou
  * error the real call would return; buf may be NULL. */
 int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, const lba_fmt* acc_fmt, int order,
                       int chunk, int is_conv, int vec_ok, char* buf, size_t buf_len);
+/* The same for lba_gemm_batched with `batch` problems (batch >= 1, else LBA_ERR_SHAPE): the tile is chosen for the
+ * CTAs of all problems together; the grid printed is that of one problem. */
+int lba_describe_plan_batched(int64_t batch, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt,
+                              const lba_fmt* acc_fmt, int order, int chunk, int is_conv, int vec_ok, char* buf,
+                              size_t buf_len);
 
 /* Testing and tuning hook: force the CTA tile (0 = 128x128, 1 = 128x64, 2 = 64x64, 3 = 32x32 outputs; 5 = the 64x64
  * tile shared by a cluster of two CTAs, each taking every second chunk, used only in chunk-16 order with floor

@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liblba.so")
 
 EXPORTS = ["lba_gemm", "lba_gemm_batched", "lba_gemm_last_overflow", "lba_gemm_ste_mask", "lba_conv2d", "lba_gemm_host_workspace_bytes", "lba_gemm_host",
-           "lba_conv2d_host_workspace_bytes", "lba_conv2d_host", "lba_gemm_host_static", "lba_count_nan_codes", "lba_describe_plan",
+           "lba_conv2d_host_workspace_bytes", "lba_conv2d_host", "lba_gemm_host_static", "lba_count_nan_codes", "lba_describe_plan", "lba_describe_plan_batched",
            "lba_set_tile_override", "lba_status_string", "lba_last_cuda_error", "lba_version"]
 
 
@@ -67,6 +67,7 @@ def load_library():
     lib.lba_count_nan_codes.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
     lib.lba_describe_plan.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.POINTER(_Fmt), C.POINTER(_Fmt), C.c_int,
                                       C.c_int, C.c_int, C.c_int, C.c_char_p, C.c_size_t]
+    lib.lba_describe_plan_batched.argtypes = [C.c_int64] + lib.lba_describe_plan.argtypes
     for name in EXPORTS:
         getattr(lib, name)
     _lib = lib
@@ -288,10 +289,12 @@ def set_tile_override(tile):
     _check(load_library().lba_set_tile_override(int(tile)))
 
 
-def describe_plan(M, N, K, prod_fmt, acc_fmt, order=ORDER_CHUNKED, chunk=PAPER_CHUNK, is_conv=False, vec_ok=True):
-    """Text description of the kernel variant a call would run; raises LbaError for rejected arguments."""
+def describe_plan(M, N, K, prod_fmt, acc_fmt, order=ORDER_CHUNKED, chunk=PAPER_CHUNK, is_conv=False, vec_ok=True, batch=1):
+    """Text description of the kernel variant a call would run (``batch`` problems for ``lba_gemm_batched``); raises
+    LbaError for rejected arguments."""
     lib = load_library()
     buf = C.create_string_buffer(256)
     pf, af = _fmt(prod_fmt), _fmt(acc_fmt)
-    _check(lib.lba_describe_plan(M, N, K, C.byref(pf), C.byref(af), order, chunk, int(is_conv), int(vec_ok), buf, 256))
+    _check(lib.lba_describe_plan_batched(batch, M, N, K, C.byref(pf), C.byref(af), order, chunk, int(is_conv), int(vec_ok),
+                                         buf, 256))
     return buf.value.decode()

@@ -826,7 +826,12 @@ int lba_count_nan_codes(const uint8_t* codes, int64_t n, unsigned long long* cou
 
 int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, const lba_fmt* acc_fmt, int order,
                       int chunk, int is_conv, int vec_ok, char* buf, size_t buf_len) {
-  if (M < 0 || N < 0 || K < 0) return LBA_ERR_SHAPE;
+  return lba_describe_plan_batched(1, M, N, K, prod_fmt, acc_fmt, order, chunk, is_conv, vec_ok, buf, buf_len);
+}
+
+int lba_describe_plan_batched(int64_t batch, int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, const lba_fmt* acc_fmt,
+                              int order, int chunk, int is_conv, int vec_ok, char* buf, size_t buf_len) {
+  if (batch < 1 || M < 0 || N < 0 || K < 0) return LBA_ERR_SHAPE;
   Plan pl;
   const int st = make_plan(prod_fmt, acc_fmt, order, chunk, K, &pl);
   if (st != LBA_OK) return st;
@@ -838,7 +843,7 @@ int lba_describe_plan(int64_t M, int64_t N, int64_t K, const lba_fmt* prod_fmt, 
     return LBA_OK;
   }
   const bool pair_ok = pl.ord == ORD_CHUNK16 && (pl.qm == QM_FLOOR_FAST || pl.qm == QM_FLOOR_FULL) && load != LD_ANY;
-  const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, 1, pl.qm, pl.ord, load, pair_ok);
+  const int tile = choose_tile(M > 0 ? M : 1, N > 0 ? N : 1, batch, pl.qm, pl.ord, load, pair_ok);
   // which kernel runs and what Q_prod costs there beyond the flush
   const bool packed = pl.ord != ORD_CHUNK_ANY &&
                       (pl.qm == QM_FLOOR_FAST || pl.qm == QM_FLOOR_FULL || (pl.qm == QM_RNE_FULL && pl.rne_packed));

@@ -114,3 +114,12 @@ def test_tile_choice_follows_the_measured_order():
     assert tile((1568, 512, 4608), f, CHK) == "tile=64x64x16 pair micro=4x8"     # layer4: two CTAs per tile
     assert tile((1568, 512, 4608), f, SEQ) == "tile=32x32x16 micro=4x4"          # no chunks to share in sequential order
     assert tile((32, 1000, 512), f, CHK) == "tile=32x32x16 micro=4x4"            # the classifier
+
+
+def test_describe_plan_for_batched_calls():
+    # 384 problems of 128x128 fill the SMs with 64x64 tiles; one such problem alone would get the 32x32 tile
+    f = code_domain_formats(7, 4)
+    assert lba.describe_plan(128, 128, 64, *f, CHK, 16).startswith("tile=32x32x16")
+    assert lba.describe_plan(128, 128, 64, *f, CHK, 16, batch=384).startswith("tile=64x64x16 micro=4x8")
+    with pytest.raises(lba.LbaError):
+        lba.describe_plan(128, 128, 64, *f, CHK, 16, batch=0)
