@@ -2,7 +2,7 @@
 host buffers, convolution, fixed point, STE masks, last overflow), formats (M, E, bias, rounding, underflow flag, input byte
 format), shapes, orders, chunk sizes, scale layouts, tile shapes and operand distributions.
 
-The number of cases of the default run is small; LBA_FUZZ_CASES and LBA_FUZZ_SEED widen it."""
+The number of cases of the default run is small; LBA_FUZZ_CASES, LBA_FUZZ_SEED and LBA_FUZZ_SCALE widen it."""
 import os
 
 import numpy as np
@@ -19,6 +19,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 CASES = int(os.environ.get("LBA_FUZZ_CASES", "400"))
 SEED = int(os.environ.get("LBA_FUZZ_SEED", "20240125"))
+SCALE = int(os.environ.get("LBA_FUZZ_SCALE", "1"))   # multiplies the largest M and N drawn (several 128-wide tiles per side)
 ERR_FORMAT = -3
 UNCHECKED = []   # cases the library ran and the oracle could not carry
 
@@ -88,7 +89,7 @@ def _one_case(rng, trial):
         acc = LbaFormat(acc.man_bits, acc.exp_bits, acc.bias, 0, acc.flags & 1)
         m4e3 = False
     small = kind in ("ste", "last", "conv")
-    M, N = int(rng.integers(1, 120 if small else 280)), int(rng.integers(1, 120 if small else 280))
+    M, N = int(rng.integers(1, (120 if small else 280) * SCALE)), int(rng.integers(1, (120 if small else 280) * SCALE))
     K = int(rng.choice([0, 1, 2, 15, 16, 17, 31, 33, 64, 100, 255, 256, 500, int(rng.integers(1, 700)), int(rng.integers(1, 700))]))
     if kind in ("gemm", "fixed", "host") and rng.random() < 0.03:     # a few long chains and wide shapes
         K = int(rng.choice([1000, 2048, 4100]))
